@@ -1,0 +1,172 @@
+/*
+ * dt8 -- fused 8-bit optimizer step over the dynamic-tree 8-bit data type (CUDA, sm_100a).
+ *
+ * C ABI of the library.  Plain pointers and sizes only; no framework types.
+ *
+ * The method is Section IV of "Memory-Efficient Training for Deep Speaker Embedding Learning
+ * in Speaker Verification" (arXiv 2412.01195): optimizer states are stored as uint8 indices into
+ * a 256-entry code book with one fp32 absolute maximum per block of B elements; a step
+ * dequantizes the states to 32-bit, applies the 32-bit SGD-momentum / Adam update to the
+ * parameters, and quantizes the new states back (Section I; Section IV-B; Eq. sgd, Eq. adam,
+ * Eq. quant1, quant2, quant3).
+ *
+ * Conventions shared by every entry point
+ *   - Return value: a dt8_status.  On any status other than DT8_OK nothing was launched and no
+ *     caller buffer was written.
+ *   - "device" pointers are CUDA device pointers of the current device, owned by the caller and
+ *     valid until the work queued on `stream` has run.  "host" pointers are ordinary host memory.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the default
+ *     stream).  They never synchronise and never allocate device memory.
+ *   - The first call on a device (or dt8_init) uploads the constant tables of the data type with
+ *     a blocking copy; make that call outside any stream capture.
+ *   - Layout: a tensor is a flat array of n elements, cut into nb = ceil(n / block_size) blocks;
+ *     block b covers elements [b*block_size, min(n, (b+1)*block_size)).  `codes` holds n bytes,
+ *     `absmax` holds nb floats (Section IV-B, "Tensor chunking").  Blocks never span tensors.
+ *   - block_size is one of 256, 512, 1024, 2048, 4096 (the paper uses 2048), else
+ *     DT8_ERR_UNSUPPORTED.
+ *   - Alignment: fp32 tensors 16 bytes, bf16 tensors 8 bytes, code arrays 4 bytes, absmax arrays
+ *     4 bytes, at each tensor's base; else DT8_ERR_ALIGNMENT.
+ *   - n == 0 (or num_tensors == 0) is a successful no-op.  n < 0, a NULL tensor pointer with
+ *     n > 0, step < 1, or an unknown dtype / flag gives DT8_ERR_INVALID_ARG.
+ *   - A state whose absmax entries are all 0 is the zero state (Eq. adam: r_0 = m_0 = 0); its code
+ *     bytes are then ignored on input.
+ *   - Codes are indices into the ASCENDING table ("the integer index i corresponding to q_i").
+ *     The signed table has two zero entries, 127 and 128; the quantizer emits 127.
+ *   - Arithmetic: everything that decides a code -- dequantized state, new state, block maximum,
+ *     normalised value -- is computed in IEEE binary32, one rounding per written operation, no
+ *     fused multiply-add, true division by the block maximum.
+ *   - Non-finite inputs are outside the contract; they cannot cause an out-of-bounds access.
+ */
+#ifndef DT8_H_
+#define DT8_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DT8_OK = 0,
+  DT8_ERR_INVALID_ARG = 1,
+  DT8_ERR_UNSUPPORTED = 2,
+  DT8_ERR_ALIGNMENT = 3,
+  DT8_ERR_CUDA = 4
+} dt8_status;
+
+/* Gradient element type. */
+typedef enum { DT8_F32 = 0, DT8_BF16 = 1 } dt8_dtype;
+
+/* Flags of dt8_adam_step.  The default used by the Python binding is both bits set (AdamW with
+ * bias correction, the optimizer the paper trains its DF-ResNets with, Section V).  With both
+ * bits clear and weight_decay = 0 the update is Eq. adam exactly as printed. */
+enum {
+  DT8_ADAM_BIAS_CORRECTION = 1, /* divide m by 1-beta1^step and r by 1-beta2^step          */
+  DT8_ADAM_DECOUPLED_WD = 2     /* w <- w(1 - lr*wd) (AdamW); clear: g <- g + wd*w (L2)     */
+};
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char *dt8_status_string(int status);
+
+/* Last CUDA error code (a cudaError_t as int) seen by a call that returned DT8_ERR_CUDA on this
+ * host thread, 0 if none. */
+int dt8_last_cuda_error(void);
+
+/*
+ * Code book of the dynamic-tree 8-bit data type (Section IV-B, "Nearest value searching",
+ * Fig. dynamic_tree): sign bit, a run of E zero bits = decimal exponent 10^-E, an indicator bit,
+ * and F fraction bits holding k, with value 10^-E * (0.1 + 0.9*(k+1)/2^F), rounded to binary32.
+ * is_signed != 0: 7-bit magnitude behind a sign bit, values in [-1, 1], used for the momentum and
+ * the Adam first moment.  is_signed == 0: 8-bit magnitude, values in [0, 1], used for the Adam
+ * second moment.  Pure host function; writes 256 ascending floats to out_host (host memory).
+ * DT8_ERR_INVALID_ARG if out_host is NULL.
+ */
+int dt8_codebook(int is_signed, float *out_host);
+
+/*
+ * Diagnostic, host only: runs the kernels' table-driven nearest-code search (the device code of
+ * Eq. quant2, compiled for the host) on n already-normalised values in host memory and writes the
+ * codes to out_host.  It exists so that the encode tables can be checked without a GPU; no step,
+ * quantize or dequantize call uses it.
+ */
+int dt8_selfcheck_encode_host(int is_signed, const float *v_host, int64_t n, uint8_t *out_host);
+
+/* Optional: upload the constant tables to the current device now (otherwise the first call does
+ * it).  Blocking; call outside stream capture. */
+int dt8_init(void);
+
+/*
+ * Block-wise quantization (Eq. quant1 + quant2).  For every block: absmax[b] = max |x_i|;
+ * v_i = x_i / absmax[b] (0 for an all-zero block); codes_i = index of the table value nearest to
+ * v_i, the lower index on an exact tie.  With the unsigned table negative inputs map to code 0.
+ *   x       device, const float[n]         input
+ *   codes   device, uint8_t[n]             output
+ *   absmax  device, float[ceil(n/B)]       output
+ */
+int dt8_quantize_blockwise(const float *x, int64_t n, int block_size, int is_signed,
+                           uint8_t *codes, float *absmax, void *stream);
+
+/*
+ * Block-wise dequantization (Eq. quant3): out_i = table[codes_i] * absmax[block of i].
+ *   codes   device, const uint8_t[n];  absmax device, const float[ceil(n/B)];  out device, float[n]
+ */
+int dt8_dequantize_blockwise(const uint8_t *codes, const float *absmax, int64_t n, int block_size,
+                             int is_signed, float *out, void *stream);
+
+/*
+ * One 8-bit SGD-with-momentum step, in place (Eq. sgd wrapped in Eq. quant3 / quant1 / quant2):
+ *     m   = table_s[m_codes] * m_absmax[b]
+ *     g'  = g + weight_decay * p                 (skipped when weight_decay == 0)
+ *     m'  = momentum * m + g'                    (from the zero state this is m_0 = g_0)
+ *     p  <- p - lr * m'
+ *     (m_codes, m_absmax) <- quantize(m') with the signed table
+ *   p         device, float[n]                   parameters, updated
+ *   g         device, const float[n] or const bf16[n] per g_dtype (bf16 is widened exactly)
+ *   m_codes   device, uint8_t[n];  m_absmax device, float[ceil(n/B)]    state, updated
+ *   step      1-based index of this step (accepted for symmetry; the rule does not use it)
+ */
+int dt8_sgd_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
+                 int64_t n, float lr, float momentum, float weight_decay, int64_t step,
+                 int block_size, void *stream);
+
+/*
+ * One 8-bit Adam / AdamW step, in place (Eq. adam wrapped in Eq. quant3 / quant1 / quant2):
+ *     m = table_s[m_codes]*m_absmax[b];  r = table_u[r_codes]*r_absmax[b]
+ *     decoupled decay: p <- p*(1 - lr*weight_decay);  coupled: g <- g + weight_decay*p
+ *     m' = beta1*m + (1-beta1)*g;   r' = beta2*r + (1-beta2)*(g*g)
+ *     p <- p - lr * (m'/bc1) / (sqrt(r'/bc2) + eps),  bc_i = 1 - beta_i^step, or 1 without bias
+ *          correction
+ *     m' is re-quantized with the signed table, r' with the unsigned table.
+ * The parameter update uses the 32-bit m', r' before they are quantized.  With decoupled decay the
+ * parameter update is evaluated with fast reciprocal / square root (relative error ~1e-7 of the
+ * update); with coupled decay, where p feeds the states, it is evaluated with IEEE operations.
+ */
+int dt8_adam_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
+                  uint8_t *r_codes, float *r_absmax, int64_t n, float lr, float beta1, float beta2,
+                  float eps, float weight_decay, int64_t step, int block_size, uint32_t flags,
+                  void *stream);
+
+/*
+ * Pointer-list forms: the same step applied to num_tensors tensors in one kernel launch per 256
+ * tensors (the paper's networks hold hundreds of small convolution and batch-norm tensors,
+ * Section III layer tables).  The arrays p, g, m_codes, m_absmax, r_codes, r_absmax and n are HOST
+ * arrays of num_tensors entries, read before the call returns; their entries are device pointers
+ * (sizes for n).  Every tensor is chunked on its own: tensor t has ceil(n[t]/B) blocks.  All
+ * gradients share g_dtype.  Tensors with n[t] == 0 are skipped.  Results are identical to calling
+ * the single-tensor form on each tensor.
+ */
+int dt8_sgd_step_multi(int num_tensors, float *const *p, const void *const *g, int g_dtype,
+                       uint8_t *const *m_codes, float *const *m_absmax, const int64_t *n, float lr,
+                       float momentum, float weight_decay, int64_t step, int block_size,
+                       void *stream);
+
+int dt8_adam_step_multi(int num_tensors, float *const *p, const void *const *g, int g_dtype,
+                        uint8_t *const *m_codes, float *const *m_absmax, uint8_t *const *r_codes,
+                        float *const *r_absmax, const int64_t *n, float lr, float beta1,
+                        float beta2, float eps, float weight_decay, int64_t step, int block_size,
+                        uint32_t flags, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DT8_H_ */

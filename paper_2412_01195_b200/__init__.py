@@ -1,0 +1,274 @@
+"""dt8: fused 8-bit optimizer step over the dynamic-tree 8-bit data type, for NVIDIA B200.
+
+Thin Python binding of the C ABI in ``include/dt8.h`` (same names, argument marshalling
+only).  Every step of the method runs in the CUDA library ``libdt8.so``; PyTorch is used for
+device memory and streams.  There is no CPU implementation behind these functions: if the
+library is missing or no CUDA device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+__all__ = [
+    "DT8Error", "lib_path", "load_library", "num_blocks",
+    "dt8_codebook", "dt8_selfcheck_encode_host", "dt8_init", "dt8_quantize_blockwise",
+    "dt8_dequantize_blockwise", "dt8_sgd_step", "dt8_adam_step", "dt8_sgd_step_multi",
+    "dt8_adam_step_multi", "new_state", "shard_blocks",
+    "DT8_F32", "DT8_BF16", "DT8_ADAM_BIAS_CORRECTION", "DT8_ADAM_DECOUPLED_WD", "DEFAULT_ADAM_FLAGS",
+    "BLOCK_SIZES",
+]
+
+DT8_OK, DT8_ERR_INVALID_ARG, DT8_ERR_UNSUPPORTED, DT8_ERR_ALIGNMENT, DT8_ERR_CUDA = range(5)
+DT8_F32, DT8_BF16 = 0, 1
+DT8_ADAM_BIAS_CORRECTION, DT8_ADAM_DECOUPLED_WD = 1, 2
+DEFAULT_ADAM_FLAGS = DT8_ADAM_BIAS_CORRECTION | DT8_ADAM_DECOUPLED_WD
+BLOCK_SIZES = (256, 512, 1024, 2048, 4096)
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdt8.so")
+_lib = None
+
+EXPORTS = (
+    "dt8_status_string", "dt8_last_cuda_error", "dt8_codebook", "dt8_selfcheck_encode_host",
+    "dt8_init", "dt8_quantize_blockwise", "dt8_dequantize_blockwise", "dt8_sgd_step",
+    "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
+)
+
+
+class DT8Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = load_library().dt8_status_string(status).decode()
+        if status == DT8_ERR_CUDA:
+            msg += " [cudaError %d]" % load_library().dt8_last_cuda_error()
+        super().__init__(f"{where}: {msg}")
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libdt8.so (built in-tree by ``paper_2412_01195_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2412_01195_b200.build` "
+            "(there is no fallback implementation)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    c = ctypes
+    vp, i64, f32, i32, u32 = c.c_void_p, c.c_int64, c.c_float, c.c_int, c.c_uint32
+    lib.dt8_status_string.restype = c.c_char_p
+    lib.dt8_status_string.argtypes = [i32]
+    lib.dt8_last_cuda_error.restype = i32
+    lib.dt8_codebook.argtypes = [i32, vp]
+    lib.dt8_selfcheck_encode_host.argtypes = [i32, vp, i64, vp]
+    lib.dt8_init.argtypes = []
+    lib.dt8_quantize_blockwise.argtypes = [vp, i64, i32, i32, vp, vp, vp]
+    lib.dt8_dequantize_blockwise.argtypes = [vp, vp, i64, i32, i32, vp, vp]
+    lib.dt8_sgd_step.argtypes = [vp, vp, i32, vp, vp, i64, f32, f32, f32, i64, i32, vp]
+    lib.dt8_adam_step.argtypes = [vp, vp, i32, vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, i32,
+                                  u32, vp]
+    lib.dt8_sgd_step_multi.argtypes = [i32, vp, vp, i32, vp, vp, vp, f32, f32, f32, i64, i32, vp]
+    lib.dt8_adam_step_multi.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, vp, f32, f32, f32, f32, f32,
+                                        i64, i32, u32, vp]
+    for name in EXPORTS:
+        getattr(lib, name).restype = getattr(lib, name).restype or i32
+    _lib = lib
+    return lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != DT8_OK:
+        raise DT8Error(status, where)
+
+
+def num_blocks(n: int, block_size: int) -> int:
+    return (n + block_size - 1) // block_size
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream], device) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream(device)
+    return s.cuda_stream
+
+
+def _dev_tensor(t: torch.Tensor, dtype, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{name}: need a contiguous CUDA tensor of dtype {dtype}")
+    return t.data_ptr()
+
+
+def _grad_ptr(g: torch.Tensor):
+    if not (isinstance(g, torch.Tensor) and g.is_cuda and g.is_contiguous()):
+        raise TypeError("g: need a contiguous CUDA tensor")
+    if g.dtype == torch.float32:
+        return g.data_ptr(), DT8_F32
+    if g.dtype == torch.bfloat16:
+        return g.data_ptr(), DT8_BF16
+    raise TypeError("g: float32 or bfloat16")
+
+
+# -----------------------------------------------------------------------------------------------
+# host-only entry points
+# -----------------------------------------------------------------------------------------------
+def dt8_codebook(is_signed: bool) -> np.ndarray:
+    """The 256 ascending values of the data type (host, no GPU needed)."""
+    out = np.empty(256, np.float32)
+    _check(load_library().dt8_codebook(int(bool(is_signed)), out.ctypes.data), "dt8_codebook")
+    return out
+
+
+def dt8_selfcheck_encode_host(is_signed: bool, v: np.ndarray) -> np.ndarray:
+    """Diagnostic: the kernels' table-driven nearest-code search run on the host."""
+    v = np.ascontiguousarray(v, np.float32).ravel()
+    out = np.empty(v.size, np.uint8)
+    _check(load_library().dt8_selfcheck_encode_host(int(bool(is_signed)), v.ctypes.data, v.size,
+                                                    out.ctypes.data), "dt8_selfcheck_encode_host")
+    return out
+
+
+# -----------------------------------------------------------------------------------------------
+# device entry points
+# -----------------------------------------------------------------------------------------------
+def dt8_init(device=None) -> None:
+    with torch.cuda.device(device if device is not None else torch.cuda.current_device()):
+        _check(load_library().dt8_init(), "dt8_init")
+
+
+def new_state(n: int, block_size: int, signed: bool, device) -> tuple:
+    """Zero state: canonical zero codes and absmax 0."""
+    codes = torch.full((n,), 127 if signed else 0, dtype=torch.uint8, device=device)
+    absmax = torch.zeros(num_blocks(n, block_size), dtype=torch.float32, device=device)
+    return codes, absmax
+
+
+def dt8_quantize_blockwise(x: torch.Tensor, block_size: int, is_signed: bool,
+                           codes: Optional[torch.Tensor] = None, absmax: Optional[torch.Tensor] = None,
+                           stream=None):
+    n = x.numel()
+    if codes is None:
+        codes = torch.empty(n, dtype=torch.uint8, device=x.device)
+    if absmax is None:
+        absmax = torch.empty(num_blocks(n, block_size), dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        st = load_library().dt8_quantize_blockwise(
+            _dev_tensor(x, torch.float32, "x"), n, block_size, int(bool(is_signed)),
+            _dev_tensor(codes, torch.uint8, "codes"), _dev_tensor(absmax, torch.float32, "absmax"),
+            _stream_ptr(stream, x.device))
+    _check(st, "dt8_quantize_blockwise")
+    return codes, absmax
+
+
+def dt8_dequantize_blockwise(codes: torch.Tensor, absmax: torch.Tensor, block_size: int,
+                             is_signed: bool, out: Optional[torch.Tensor] = None, stream=None):
+    n = codes.numel()
+    if out is None:
+        out = torch.empty(n, dtype=torch.float32, device=codes.device)
+    with torch.cuda.device(codes.device):
+        st = load_library().dt8_dequantize_blockwise(
+            _dev_tensor(codes, torch.uint8, "codes"), _dev_tensor(absmax, torch.float32, "absmax"), n,
+            block_size, int(bool(is_signed)), _dev_tensor(out, torch.float32, "out"),
+            _stream_ptr(stream, codes.device))
+    _check(st, "dt8_dequantize_blockwise")
+    return out
+
+
+def dt8_sgd_step(p, g, m_codes, m_absmax, lr, momentum, weight_decay, step, block_size=2048,
+                 stream=None) -> None:
+    gp, gd = _grad_ptr(g)
+    with torch.cuda.device(p.device):
+        st = load_library().dt8_sgd_step(
+            _dev_tensor(p, torch.float32, "p"), gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
+            _dev_tensor(m_absmax, torch.float32, "m_absmax"), p.numel(), lr, momentum, weight_decay,
+            step, block_size, _stream_ptr(stream, p.device))
+    _check(st, "dt8_sgd_step")
+
+
+def dt8_adam_step(p, g, m_codes, m_absmax, r_codes, r_absmax, lr, beta1, beta2, eps, weight_decay,
+                  step, block_size=2048, flags=DEFAULT_ADAM_FLAGS, stream=None) -> None:
+    gp, gd = _grad_ptr(g)
+    with torch.cuda.device(p.device):
+        st = load_library().dt8_adam_step(
+            _dev_tensor(p, torch.float32, "p"), gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
+            _dev_tensor(m_absmax, torch.float32, "m_absmax"), _dev_tensor(r_codes, torch.uint8, "r_codes"),
+            _dev_tensor(r_absmax, torch.float32, "r_absmax"), p.numel(), lr, beta1, beta2, eps,
+            weight_decay, step, block_size, flags, _stream_ptr(stream, p.device))
+    _check(st, "dt8_adam_step")
+
+
+class _PtrList:
+    """Host arrays of device pointers / sizes for the pointer-list entry points."""
+
+    def __init__(self, tensors: Sequence[torch.Tensor], dtype, name: str):
+        self.arr = (ctypes.c_void_p * len(tensors))(*[_dev_tensor(t, dtype, name) for t in tensors])
+
+    @property
+    def ptr(self):
+        return ctypes.cast(self.arr, ctypes.c_void_p)
+
+
+def _multi_common(ps, gs):
+    if len(ps) == 0:
+        return None, None, None, None
+    dev = ps[0].device
+    gdt = gs[0].dtype
+    if any(g.dtype != gdt for g in gs):
+        raise TypeError("all gradients of one call share a dtype")
+    _, gd = _grad_ptr(gs[0])
+    garr = (ctypes.c_void_p * len(gs))(*[_grad_ptr(g)[0] for g in gs])
+    narr = (ctypes.c_int64 * len(ps))(*[p.numel() for p in ps])
+    return dev, gd, garr, narr
+
+
+def dt8_sgd_step_multi(ps, gs, m_codes, m_absmax, lr, momentum, weight_decay, step, block_size=2048,
+                       stream=None) -> None:
+    dev, gd, garr, narr = _multi_common(ps, gs)
+    if dev is None:
+        return
+    pl = _PtrList(ps, torch.float32, "p")
+    mc = _PtrList(m_codes, torch.uint8, "m_codes")
+    ma = _PtrList(m_absmax, torch.float32, "m_absmax")
+    with torch.cuda.device(dev):
+        st = load_library().dt8_sgd_step_multi(
+            len(ps), pl.ptr, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr,
+            ctypes.cast(narr, ctypes.c_void_p), lr, momentum, weight_decay, step, block_size,
+            _stream_ptr(stream, dev))
+    _check(st, "dt8_sgd_step_multi")
+
+
+def dt8_adam_step_multi(ps, gs, m_codes, m_absmax, r_codes, r_absmax, lr, beta1, beta2, eps,
+                        weight_decay, step, block_size=2048, flags=DEFAULT_ADAM_FLAGS, stream=None) -> None:
+    dev, gd, garr, narr = _multi_common(ps, gs)
+    if dev is None:
+        return
+    pl = _PtrList(ps, torch.float32, "p")
+    mc = _PtrList(m_codes, torch.uint8, "m_codes")
+    ma = _PtrList(m_absmax, torch.float32, "m_absmax")
+    rc = _PtrList(r_codes, torch.uint8, "r_codes")
+    ra = _PtrList(r_absmax, torch.float32, "r_absmax")
+    with torch.cuda.device(dev):
+        st = load_library().dt8_adam_step_multi(
+            len(ps), pl.ptr, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr, rc.ptr, ra.ptr,
+            ctypes.cast(narr, ctypes.c_void_p), lr, beta1, beta2, eps, weight_decay, step, block_size,
+            flags, _stream_ptr(stream, dev))
+    _check(st, "dt8_adam_step_multi")
+
+
+def shard_blocks(num_blocks_total: int, rank: int, world_size: int) -> range:
+    """Contiguous range of whole quantization blocks owned by `rank`.
+
+    Blocks are independent (Section IV-B, "quantization applied independently to each block"),
+    so a tensor can be split across ranks on block boundaries with no exchange between them.
+    The first `num_blocks_total % world_size` ranks own one extra block."""
+    if not (0 <= rank < world_size):
+        raise ValueError("rank out of range")
+    q, r = divmod(num_blocks_total, world_size)
+    start = rank * q + min(rank, r)
+    return range(start, start + q + (1 if rank < r else 0))

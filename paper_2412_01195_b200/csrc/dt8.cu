@@ -1,0 +1,455 @@
+// C ABI of the dt8 library: argument checks, table upload, kernel selection and launch.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "dt8.h"
+#include "dt8_kernels.cuh"
+
+namespace dt8 {
+
+
+namespace {
+
+thread_local int tl_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e) {
+  tl_last_cuda_error = static_cast<int>(e);
+  return DT8_ERR_CUDA;
+}
+
+constexpr int kMaxDevices = 64;
+
+struct DeviceInfo {
+  int device = -1;
+  int sm_count = 0;
+};
+
+std::mutex g_init_mutex;
+std::atomic<bool> g_uploaded[kMaxDevices];
+int g_sm_count[kMaxDevices];
+
+// Makes sure the current device holds the constant tables; returns the device's SM count.
+int ensure_device(DeviceInfo* info, EncMeta* em) {
+  const Tables* ht = host_tables();
+  if (!ht) return DT8_ERR_UNSUPPORTED;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return DT8_ERR_UNSUPPORTED;
+  if (!g_uploaded[dev].load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_init_mutex);
+    if (!g_uploaded[dev].load(std::memory_order_relaxed)) {
+      static DeviceTables staging;  // guarded by g_init_mutex
+      std::memcpy(staging.dec_s, ht->dec_signed, sizeof(staging.dec_s));
+      std::memcpy(staging.dec_u, ht->dec_unsigned, sizeof(staging.dec_u));
+      std::memset(staging.enc_s, 0, sizeof(staging.enc_s));
+      std::memset(staging.enc_u, 0, sizeof(staging.enc_u));
+      std::memcpy(staging.enc_s, ht->enc_signed.entries, sizeof(uint32_t) * ht->enc_signed.num_entries);
+      std::memcpy(staging.enc_u, ht->enc_unsigned.entries, sizeof(uint32_t) * ht->enc_unsigned.num_entries);
+      e = cudaMemcpyToSymbol(g_tables, &staging, sizeof(staging));
+      if (e != cudaSuccess) return cuda_fail(e);
+      int sms = 0;
+      e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      if (e != cudaSuccess) return cuda_fail(e);
+      g_sm_count[dev] = sms;
+      g_uploaded[dev].store(true, std::memory_order_release);
+    }
+  }
+  info->device = dev;
+  info->sm_count = g_sm_count[dev];
+  em->s_first = ht->enc_signed.first_key;
+  em->u_first = ht->enc_unsigned.first_key;
+  em->s_n = ht->enc_signed.num_entries;
+  em->u_n = ht->enc_unsigned.num_entries;
+  return DT8_OK;
+}
+
+// Opt a kernel in to its dynamic shared memory size, once per device.
+template <class K>
+cudaError_t allow_smem(K kernel, int device, size_t bytes) {
+  static std::atomic<uint64_t> done{0};
+  const uint64_t bit = 1ull << device;
+  if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(bytes));
+  if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+bool block_size_ok(int B) { return B == 256 || B == 512 || B == 1024 || B == 2048 || B == 4096; }
+
+int log2_int(int v) {
+  int s = 0;
+  while ((1 << s) < v) ++s;
+  return s;
+}
+
+int grid_for(int64_t blocks, int groups_per_cta, int sm_count) {
+  const int64_t want = (blocks + groups_per_cta - 1) / groups_per_cta;
+  return static_cast<int>(want < sm_count ? want : sm_count);
+}
+
+// Values per thread for each supported block size.
+template <int B> struct Geometry { static constexpr int VPT = 8; };
+
+
+int check_tensor(const TensorDesc& d, int g_dtype, bool adam) {
+  if (d.n < 0) return DT8_ERR_INVALID_ARG;
+  if (d.n == 0) return DT8_OK;
+  if (!d.p || !d.g || !d.mc || !d.ma) return DT8_ERR_INVALID_ARG;
+  if (adam && (!d.rc || !d.ra)) return DT8_ERR_INVALID_ARG;
+  if (!aligned(d.p, 16) || !aligned(d.g, g_dtype == DT8_F32 ? 16 : 8) || !aligned(d.mc, 4) ||
+      !aligned(d.ma, 4))
+    return DT8_ERR_ALIGNMENT;
+  if (adam && (!aligned(d.rc, 4) || !aligned(d.ra, 4))) return DT8_ERR_ALIGNMENT;
+  return DT8_OK;
+}
+
+// ---- launchers -------------------------------------------------------------------------------
+template <class Args, int B, bool GBF16, bool EXACT>
+int launch_adam(const Args& args, int64_t blocks, const AdamHyper& h, const EncMeta& em,
+                const DeviceInfo& di, cudaStream_t stream) {
+  constexpr int VPT = Geometry<B>::VPT;
+  constexpr int GROUPS = kCtaThreads / (B / VPT);
+  auto kernel = adam_kernel<Args, B, VPT, GBF16, EXACT>;
+  const size_t smem = smem_bytes(em, true, true, true, true);
+  cudaError_t e = allow_smem(kernel, di.device, smem);
+  if (e != cudaSuccess) return cuda_fail(e);
+  kernel<<<grid_for(blocks, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(args, h, em);
+  e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
+template <class Args, int B>
+int dispatch_adam(const Args& args, int64_t blocks, int g_dtype, bool exact, const AdamHyper& h,
+                  const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
+  if (g_dtype == DT8_BF16)
+    return exact ? launch_adam<Args, B, true, true>(args, blocks, h, em, di, s)
+                 : launch_adam<Args, B, true, false>(args, blocks, h, em, di, s);
+  return exact ? launch_adam<Args, B, false, true>(args, blocks, h, em, di, s)
+               : launch_adam<Args, B, false, false>(args, blocks, h, em, di, s);
+}
+
+template <class Args>
+int dispatch_adam_b(const Args& args, int64_t blocks, int B, int g_dtype, bool exact,
+                    const AdamHyper& h, const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
+  switch (B) {
+    case 256: return dispatch_adam<Args, 256>(args, blocks, g_dtype, exact, h, em, di, s);
+    case 512: return dispatch_adam<Args, 512>(args, blocks, g_dtype, exact, h, em, di, s);
+    case 1024: return dispatch_adam<Args, 1024>(args, blocks, g_dtype, exact, h, em, di, s);
+    case 2048: return dispatch_adam<Args, 2048>(args, blocks, g_dtype, exact, h, em, di, s);
+    case 4096: return dispatch_adam<Args, 4096>(args, blocks, g_dtype, exact, h, em, di, s);
+  }
+  return DT8_ERR_UNSUPPORTED;
+}
+
+template <class Args, int B, bool GBF16>
+int launch_sgd(const Args& args, int64_t blocks, const SgdHyper& h, const EncMeta& em,
+               const DeviceInfo& di, cudaStream_t stream) {
+  constexpr int VPT = Geometry<B>::VPT;
+  constexpr int GROUPS = kCtaThreads / (B / VPT);
+  auto kernel = sgd_kernel<Args, B, VPT, GBF16>;
+  const size_t smem = smem_bytes(em, true, false, true, true);
+  cudaError_t e = allow_smem(kernel, di.device, smem);
+  if (e != cudaSuccess) return cuda_fail(e);
+  kernel<<<grid_for(blocks, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(args, h, em);
+  e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
+template <class Args>
+int dispatch_sgd_b(const Args& args, int64_t blocks, int B, int g_dtype, const SgdHyper& h,
+                   const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
+#define DT8_SGD_CASE(BS)                                                        \
+  case BS:                                                                      \
+    return g_dtype == DT8_BF16 ? launch_sgd<Args, BS, true>(args, blocks, h, em, di, s) \
+                               : launch_sgd<Args, BS, false>(args, blocks, h, em, di, s);
+  switch (B) {
+    DT8_SGD_CASE(256)
+    DT8_SGD_CASE(512)
+    DT8_SGD_CASE(1024)
+    DT8_SGD_CASE(2048)
+    DT8_SGD_CASE(4096)
+  }
+#undef DT8_SGD_CASE
+  return DT8_ERR_UNSUPPORTED;
+}
+
+template <int B, bool SIGNED>
+int launch_quantize(const float* x, int64_t n, uint8_t* codes, float* absmax, const EncMeta& em,
+                    const DeviceInfo& di, cudaStream_t stream) {
+  constexpr int VPT = Geometry<B>::VPT;
+  constexpr int GROUPS = kCtaThreads / (B / VPT);
+  auto kernel = quantize_kernel<B, VPT, SIGNED>;
+  const size_t smem = smem_bytes(em, SIGNED, !SIGNED, false, true);
+  cudaError_t e = allow_smem(kernel, di.device, smem);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const int64_t nb = (n + B - 1) / B;
+  kernel<<<grid_for(nb, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(x, codes, absmax, n, nb, em);
+  e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
+AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float wd, int64_t step,
+                          uint32_t flags) {
+  AdamHyper h;
+  h.beta1 = beta1;
+  h.beta2 = beta2;
+  h.omb1 = 1.0f - beta1;
+  h.omb2 = 1.0f - beta2;
+  h.lr = lr;
+  h.eps = eps;
+  h.wd = wd;
+  h.decay = 1.0f - lr * wd;
+  if (flags & DT8_ADAM_BIAS_CORRECTION) {
+    h.bc1 = static_cast<float>(1.0 - std::pow(static_cast<double>(beta1), static_cast<double>(step)));
+    h.bc2 = static_cast<float>(1.0 - std::pow(static_cast<double>(beta2), static_cast<double>(step)));
+  } else {
+    h.bc1 = 1.0f;
+    h.bc2 = 1.0f;
+  }
+  h.step_scale = lr / h.bc1;
+  h.ibc2 = 1.0f / h.bc2;
+  return h;
+}
+
+}  // namespace
+}  // namespace dt8
+
+using namespace dt8;
+
+extern "C" {
+
+const char* dt8_status_string(int status) {
+  switch (status) {
+    case DT8_OK: return "DT8_OK";
+    case DT8_ERR_INVALID_ARG: return "DT8_ERR_INVALID_ARG: bad pointer, size, step, dtype or flag";
+    case DT8_ERR_UNSUPPORTED: return "DT8_ERR_UNSUPPORTED: block size must be 256, 512, 1024, 2048 or 4096";
+    case DT8_ERR_ALIGNMENT: return "DT8_ERR_ALIGNMENT: fp32 tensors need 16-byte, bf16 8-byte, codes and absmax 4-byte alignment";
+    case DT8_ERR_CUDA: return "DT8_ERR_CUDA: a CUDA runtime call failed (see dt8_last_cuda_error)";
+  }
+  return "unknown dt8 status";
+}
+
+int dt8_last_cuda_error(void) { return tl_last_cuda_error; }
+
+int dt8_codebook(int is_signed, float* out_host) {
+  if (!out_host) return DT8_ERR_INVALID_ARG;
+  build_codebook(is_signed != 0, out_host);
+  return DT8_OK;
+}
+
+int dt8_selfcheck_encode_host(int is_signed, const float* v_host, int64_t n, uint8_t* out_host) {
+  if (n < 0 || (n > 0 && (!v_host || !out_host))) return DT8_ERR_INVALID_ARG;
+  const Tables* ht = host_tables();
+  if (!ht) return DT8_ERR_UNSUPPORTED;
+  const EncTable& e = is_signed ? ht->enc_signed : ht->enc_unsigned;
+  for (int64_t i = 0; i < n; ++i) {
+    uint32_t bits;
+    std::memcpy(&bits, v_host + i, 4);
+    out_host[i] = static_cast<uint8_t>(is_signed ? encode_signed(e.entries, e.first_key, e.num_entries, bits)
+                                                 : encode_unsigned(e.entries, e.first_key, e.num_entries, bits));
+  }
+  return DT8_OK;
+}
+
+int dt8_init(void) {
+  DeviceInfo di;
+  EncMeta em;
+  return ensure_device(&di, &em);
+}
+
+int dt8_quantize_blockwise(const float* x, int64_t n, int block_size, int is_signed, uint8_t* codes,
+                           float* absmax, void* stream) {
+  if (n < 0) return DT8_ERR_INVALID_ARG;
+  if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
+  if (n == 0) return DT8_OK;
+  if (!x || !codes || !absmax) return DT8_ERR_INVALID_ARG;
+  if (!aligned(x, 16) || !aligned(codes, 4) || !aligned(absmax, 4)) return DT8_ERR_ALIGNMENT;
+  DeviceInfo di;
+  EncMeta em;
+  int rc = ensure_device(&di, &em);
+  if (rc != DT8_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+#define DT8_Q_CASE(BS)                                                                  \
+  case BS:                                                                              \
+    return is_signed ? launch_quantize<BS, true>(x, n, codes, absmax, em, di, s)        \
+                     : launch_quantize<BS, false>(x, n, codes, absmax, em, di, s);
+  switch (block_size) {
+    DT8_Q_CASE(256)
+    DT8_Q_CASE(512)
+    DT8_Q_CASE(1024)
+    DT8_Q_CASE(2048)
+    DT8_Q_CASE(4096)
+  }
+#undef DT8_Q_CASE
+  return DT8_ERR_UNSUPPORTED;
+}
+
+int dt8_dequantize_blockwise(const uint8_t* codes, const float* absmax, int64_t n, int block_size,
+                             int is_signed, float* out, void* stream) {
+  if (n < 0) return DT8_ERR_INVALID_ARG;
+  if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
+  if (n == 0) return DT8_OK;
+  if (!codes || !absmax || !out) return DT8_ERR_INVALID_ARG;
+  if (!aligned(out, 16) || !aligned(codes, 4) || !aligned(absmax, 4)) return DT8_ERR_ALIGNMENT;
+  DeviceInfo di;
+  EncMeta em;
+  int rc = ensure_device(&di, &em);
+  if (rc != DT8_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t quads = (n + 3) / 4;
+  const int64_t ctas = (quads + kCtaThreads - 1) / kCtaThreads;
+  const int grid = static_cast<int>(ctas < 2 * di.sm_count ? ctas : 2 * di.sm_count);
+  const int shift = log2_int(block_size);
+  cudaError_t e;
+  if (is_signed) {
+    const size_t smem = smem_bytes(em, true, false, true, false);
+    e = allow_smem(dequantize_kernel<true>, di.device, smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+    dequantize_kernel<true><<<grid, kCtaThreads, smem, s>>>(codes, absmax, out, n, shift, em);
+  } else {
+    const size_t smem = smem_bytes(em, false, true, true, false);
+    e = allow_smem(dequantize_kernel<false>, di.device, smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+    dequantize_kernel<false><<<grid, kCtaThreads, smem, s>>>(codes, absmax, out, n, shift, em);
+  }
+  e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
+int dt8_sgd_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float* m_absmax, int64_t n,
+                 float lr, float momentum, float weight_decay, int64_t step, int block_size,
+                 void* stream) {
+  if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
+  if (step < 1) return DT8_ERR_INVALID_ARG;
+  if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
+  SingleArgs a;
+  a.t = TensorDesc{p, g, m_codes, m_absmax, nullptr, nullptr, n};
+  int rc = check_tensor(a.t, g_dtype, false);
+  if (rc != DT8_OK || n == 0) return rc;
+  a.nb = (n + block_size - 1) / block_size;
+  DeviceInfo di;
+  EncMeta em;
+  rc = ensure_device(&di, &em);
+  if (rc != DT8_OK) return rc;
+  const SgdHyper h{lr, momentum, weight_decay};
+  return dispatch_sgd_b(a, a.nb, block_size, g_dtype, h, em, di, static_cast<cudaStream_t>(stream));
+}
+
+int dt8_adam_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float* m_absmax,
+                  uint8_t* r_codes, float* r_absmax, int64_t n, float lr, float beta1, float beta2,
+                  float eps, float weight_decay, int64_t step, int block_size, uint32_t flags,
+                  void* stream) {
+  if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
+  if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
+  if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
+  SingleArgs a;
+  a.t = TensorDesc{p, g, m_codes, m_absmax, r_codes, r_absmax, n};
+  int rc = check_tensor(a.t, g_dtype, true);
+  if (rc != DT8_OK || n == 0) return rc;
+  a.nb = (n + block_size - 1) / block_size;
+  DeviceInfo di;
+  EncMeta em;
+  rc = ensure_device(&di, &em);
+  if (rc != DT8_OK) return rc;
+  const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
+  const bool exact = !(flags & DT8_ADAM_DECOUPLED_WD);
+  return dispatch_adam_b(a, a.nb, block_size, g_dtype, exact, h, em, di,
+                         static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"
+
+namespace dt8 {
+namespace {
+
+// Shared front end of the two pointer-list entry points: validates every tensor first (so that a
+// bad entry means nothing was launched), then launches one kernel per kMaxTensorsPerLaunch
+// non-empty tensors.
+template <class Launch>
+int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtype,
+              uint8_t* const* mc, float* const* ma, uint8_t* const* rc, float* const* ra,
+              const int64_t* n, int block_size, bool adam, Launch launch) {
+  if (num_tensors < 0) return DT8_ERR_INVALID_ARG;
+  if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
+  if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
+  if (num_tensors == 0) return DT8_OK;
+  if (!p || !g || !mc || !ma || !n || (adam && (!rc || !ra))) return DT8_ERR_INVALID_ARG;
+  for (int i = 0; i < num_tensors; ++i) {
+    const TensorDesc d{p[i], g[i], mc[i], ma[i], adam ? rc[i] : nullptr, adam ? ra[i] : nullptr, n[i]};
+    const int st = check_tensor(d, g_dtype, adam);
+    if (st != DT8_OK) return st;
+    if ((n[i] + block_size - 1) / block_size > 0x3FFFFFFF) return DT8_ERR_UNSUPPORTED;
+  }
+  DeviceInfo di;
+  EncMeta em;
+  int st = ensure_device(&di, &em);
+  if (st != DT8_OK) return st;
+  static thread_local MultiArgs args;
+  int i = 0;
+  while (i < num_tensors) {
+    args.num = 0;
+    args.blk_start[0] = 0;
+    int64_t blocks = 0;
+    while (i < num_tensors && args.num < kMaxTensorsPerLaunch) {
+      if (n[i] > 0) {
+        const int64_t nb = (n[i] + block_size - 1) / block_size;
+        if (blocks + nb > 0x7FFFFFFF) {
+          if (args.num == 0) return DT8_ERR_UNSUPPORTED;
+          break;
+        }
+        args.t[args.num] = TensorDesc{p[i], g[i], mc[i], ma[i], adam ? rc[i] : nullptr,
+                                      adam ? ra[i] : nullptr, n[i]};
+        blocks += nb;
+        args.blk_start[++args.num] = static_cast<int>(blocks);
+      }
+      ++i;
+    }
+    if (args.num == 0) continue;
+    st = launch(args, blocks, em, di);
+    if (st != DT8_OK) return st;
+  }
+  return DT8_OK;
+}
+
+}  // namespace
+}  // namespace dt8
+
+extern "C" {
+
+int dt8_sgd_step_multi(int num_tensors, float* const* p, const void* const* g, int g_dtype,
+                       uint8_t* const* m_codes, float* const* m_absmax, const int64_t* n, float lr,
+                       float momentum, float weight_decay, int64_t step, int block_size,
+                       void* stream) {
+  if (step < 1) return DT8_ERR_INVALID_ARG;
+  const SgdHyper h{lr, momentum, weight_decay};
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  return run_multi(num_tensors, p, g, g_dtype, m_codes, m_absmax, nullptr, nullptr, n, block_size,
+                   false, [&](const MultiArgs& a, int64_t blocks, const EncMeta& em, const DeviceInfo& di) {
+                     return dispatch_sgd_b(a, blocks, block_size, g_dtype, h, em, di, s);
+                   });
+}
+
+int dt8_adam_step_multi(int num_tensors, float* const* p, const void* const* g, int g_dtype,
+                        uint8_t* const* m_codes, float* const* m_absmax, uint8_t* const* r_codes,
+                        float* const* r_absmax, const int64_t* n, float lr, float beta1, float beta2,
+                        float eps, float weight_decay, int64_t step, int block_size, uint32_t flags,
+                        void* stream) {
+  if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
+  const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
+  const bool exact = !(flags & DT8_ADAM_DECOUPLED_WD);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  return run_multi(num_tensors, p, g, g_dtype, m_codes, m_absmax, r_codes, r_absmax, n, block_size,
+                   true, [&](const MultiArgs& a, int64_t blocks, const EncMeta& em, const DeviceInfo& di) {
+                     return dispatch_adam_b(a, blocks, block_size, g_dtype, exact, h, em, di, s);
+                   });
+}
+
+}  // extern "C"

@@ -1,0 +1,179 @@
+"""CPU-side checks of the CUDA library: it loads, exports what include/dt8.h declares, rejects bad
+arguments before touching a device, and its host-built tables agree with the CPU checker.
+No compute call reaches a GPU here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2412_01195_b200 as dt8
+from paper_2412_01195_b200 import build as dt8_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    dt8_build.build_library()
+    return dt8.load_library()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "dt8.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dt8_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_symbols()
+    assert {"dt8_codebook", "dt8_quantize_blockwise", "dt8_dequantize_blockwise", "dt8_sgd_step",
+            "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(dt8.EXPORTS)
+
+
+def test_status_strings(lib):
+    for code in range(5):
+        assert lib.dt8_status_string(code).decode().startswith("DT8_")
+    assert b"unknown" in lib.dt8_status_string(99)
+
+
+@pytest.mark.parametrize("signed", [True, False])
+def test_codebook_is_bit_identical_to_the_checker(signed):
+    a, b = dt8.dt8_codebook(signed), oracle.codebook(signed)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_codebook_null(lib):
+    assert lib.dt8_codebook(1, None) == dt8.DT8_ERR_INVALID_ARG
+
+
+def ulp_neighbourhood(x32, radius):
+    bits = x32.astype(np.float32).view(np.int32).astype(np.int64)
+    return np.concatenate([(bits + d).astype(np.int32).view(np.float32) for d in range(-radius, radius + 1)])
+
+
+@pytest.mark.parametrize("signed", [True, False])
+def test_table_encoder_equals_checker_on_critical_inputs(signed):
+    Q = oracle.codebook(signed)
+    Q64 = Q.astype(np.float64)
+    mids = ((Q64[:-1] + Q64[1:]) / 2).astype(np.float32)
+    rng = np.random.default_rng(70)
+    pools = [Q, ulp_neighbourhood(Q, 8), ulp_neighbourhood(mids, 64), -ulp_neighbourhood(mids, 64),
+             rng.uniform(-1, 1, 1_000_000).astype(np.float32),
+             (10.0 ** rng.uniform(-12, 0, 500_000) * rng.choice([-1, 1], 500_000)).astype(np.float32),
+             np.array([0.0, -0.0, 1.0, -1.0, 1e-38, -1e-38, 1e-45, 2.0, -2.0, 1e30, -1e30], np.float32)]
+    for v in pools:
+        v = v[np.isfinite(v)]
+        assert np.array_equal(dt8.dt8_selfcheck_encode_host(signed, v), oracle.nearest(Q, v))
+    # bucket edges of the table: all values whose low 15/16 bits are 0, 1 or all-ones
+    expo = np.arange(90, 128, dtype=np.uint32)[:, None, None] << 23
+    mant_hi = (np.arange(256, dtype=np.uint32) << 15)[None, :, None]
+    low = np.array([0, 1, 2, 0x7FFE, 0x7FFF], np.uint32)[None, None, :]
+    edge = (expo | mant_hi | low).ravel().view(np.float32)
+    edge = np.concatenate([edge, -edge])
+    assert np.array_equal(dt8.dt8_selfcheck_encode_host(signed, edge), oracle.nearest(Q, edge))
+
+
+@pytest.mark.parametrize("signed", [True, False])
+def test_table_encoder_strided_sweep_of_all_floats(signed):
+    """Every 61st binary32 bit pattern with |v| <= 1, both signs (about 35 million values)."""
+    Q = oracle.codebook(signed)
+    bits = np.arange(0, 0x3F800001, 61, dtype=np.uint32)
+    for sign in (0, 0x80000000):
+        v = (bits | np.uint32(sign)).view(np.float32)
+        assert np.array_equal(dt8.dt8_selfcheck_encode_host(signed, v), oracle.nearest(Q, v))
+
+
+def test_non_finite_inputs_stay_inside_the_tables():
+    v = np.array([np.nan, -np.nan, np.inf, -np.inf, 3e38, -3e38], np.float32)
+    for signed in (True, False):
+        dt8.dt8_selfcheck_encode_host(signed, v)      # must not crash; values unspecified
+
+
+def test_argument_checks_return_before_any_device_work(lib):
+    """These all fail validation on the host, so they are safe without a GPU."""
+    f = lambda x: ctypes.c_float(x)
+    buf = (ctypes.c_uint8 * 4096)()
+    base = ctypes.addressof(buf)
+    base += (-base) % 16
+    ok, odd = ctypes.c_void_p(base), ctypes.c_void_p(base + 2)
+    E = dt8
+    # bad block size / sizes / null pointers / alignment for quantize and dequantize
+    assert lib.dt8_quantize_blockwise(ok, 16, 1000, 1, ok, ok, None) == E.DT8_ERR_UNSUPPORTED
+    assert lib.dt8_quantize_blockwise(ok, -1, 2048, 1, ok, ok, None) == E.DT8_ERR_INVALID_ARG
+    assert lib.dt8_quantize_blockwise(None, 16, 2048, 1, ok, ok, None) == E.DT8_ERR_INVALID_ARG
+    assert lib.dt8_quantize_blockwise(odd, 16, 2048, 1, ok, ok, None) == E.DT8_ERR_ALIGNMENT
+    assert lib.dt8_quantize_blockwise(ok, 0, 2048, 1, None, None, None) == E.DT8_OK
+    assert lib.dt8_dequantize_blockwise(ok, ok, 16, 300, 0, ok, None) == E.DT8_ERR_UNSUPPORTED
+    assert lib.dt8_dequantize_blockwise(ok, None, 16, 256, 0, ok, None) == E.DT8_ERR_INVALID_ARG
+    assert lib.dt8_dequantize_blockwise(ok, ok, 16, 256, 0, odd, None) == E.DT8_ERR_ALIGNMENT
+    assert lib.dt8_dequantize_blockwise(None, None, 0, 256, 0, None, None) == E.DT8_OK
+    # sgd
+    sgd = lambda p, g, gd, mc, ma, n, step, B: lib.dt8_sgd_step(p, g, gd, mc, ma, n, f(.1), f(.9), f(0), step, B, None)
+    assert sgd(ok, ok, 7, ok, ok, 16, 1, 2048) == E.DT8_ERR_INVALID_ARG
+    assert sgd(ok, ok, 0, ok, ok, 16, 0, 2048) == E.DT8_ERR_INVALID_ARG
+    assert sgd(ok, ok, 0, ok, ok, -5, 1, 2048) == E.DT8_ERR_INVALID_ARG
+    assert sgd(ok, ok, 0, ok, ok, 16, 1, 100) == E.DT8_ERR_UNSUPPORTED
+    assert sgd(None, ok, 0, ok, ok, 16, 1, 2048) == E.DT8_ERR_INVALID_ARG
+    assert sgd(odd, ok, 0, ok, ok, 16, 1, 2048) == E.DT8_ERR_ALIGNMENT
+    assert sgd(ok, ok, 0, odd, ok, 16, 1, 2048) == E.DT8_ERR_ALIGNMENT
+    assert sgd(None, None, 0, None, None, 0, 1, 2048) == E.DT8_OK
+    # adam
+    adam = lambda p, g, gd, mc, ma, rc, ra, n, step, B, fl: lib.dt8_adam_step(
+        p, g, gd, mc, ma, rc, ra, n, f(1e-3), f(.9), f(.999), f(1e-8), f(0), step, B, fl, None)
+    assert adam(ok, ok, 0, ok, ok, ok, ok, 16, 1, 2048, 8) == E.DT8_ERR_INVALID_ARG
+    assert adam(ok, ok, 0, ok, ok, ok, ok, 16, 0, 2048, 3) == E.DT8_ERR_INVALID_ARG
+    assert adam(ok, ok, 2, ok, ok, ok, ok, 16, 1, 2048, 3) == E.DT8_ERR_INVALID_ARG
+    assert adam(ok, ok, 0, ok, ok, None, ok, 16, 1, 2048, 3) == E.DT8_ERR_INVALID_ARG
+    assert adam(ok, ok, 0, ok, ok, ok, odd, 16, 1, 2048, 3) == E.DT8_ERR_ALIGNMENT
+    assert adam(ok, ok, 0, ok, ok, ok, ok, 16, 1, 4000, 3) == E.DT8_ERR_UNSUPPORTED
+    assert adam(None, None, 0, None, None, None, None, 0, 1, 2048, 3) == E.DT8_OK
+    # bf16 gradients need only 8-byte alignment
+    half = ctypes.c_void_p(base + 8)
+    assert adam(ok, half, 0, ok, ok, ok, ok, 16, 1, 2048, 3) == E.DT8_ERR_ALIGNMENT
+    # pointer lists
+    arr = (ctypes.c_void_p * 2)(base, base)
+    bad = (ctypes.c_void_p * 2)(base, base + 2)
+    ns = (ctypes.c_int64 * 2)(16, 16)
+    neg = (ctypes.c_int64 * 2)(16, -1)
+    ap, bp = ctypes.cast(arr, ctypes.c_void_p), ctypes.cast(bad, ctypes.c_void_p)
+    nsp, negp = ctypes.cast(ns, ctypes.c_void_p), ctypes.cast(neg, ctypes.c_void_p)
+    sgdm = lambda num, p, n, B=2048, step=1: lib.dt8_sgd_step_multi(num, p, ap, 0, ap, ap, n, f(.1), f(.9), f(0), step, B, None)
+    assert sgdm(-1, ap, nsp) == E.DT8_ERR_INVALID_ARG
+    assert sgdm(0, None, None) == E.DT8_OK
+    assert sgdm(2, None, nsp) == E.DT8_ERR_INVALID_ARG
+    assert sgdm(2, bp, nsp) == E.DT8_ERR_ALIGNMENT
+    assert sgdm(2, ap, negp) == E.DT8_ERR_INVALID_ARG
+    assert sgdm(2, ap, nsp, B=77) == E.DT8_ERR_UNSUPPORTED
+    assert sgdm(2, ap, nsp, step=0) == E.DT8_ERR_INVALID_ARG
+    adamm = lambda num, p, rc, n, fl=3: lib.dt8_adam_step_multi(
+        num, p, ap, 0, ap, ap, rc, ap, n, f(1e-3), f(.9), f(.999), f(1e-8), f(0), 1, 2048, fl, None)
+    assert adamm(2, ap, None, nsp) == E.DT8_ERR_INVALID_ARG
+    assert adamm(2, ap, bp, nsp) == E.DT8_ERR_ALIGNMENT
+    assert adamm(2, ap, ap, nsp, fl=4) == E.DT8_ERR_INVALID_ARG
+    assert adamm(0, None, None, None) == E.DT8_OK
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(dt8, "_lib", None)
+    monkeypatch.setattr(dt8, "_LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        dt8.dt8_codebook(True)
+
+
+def test_shard_blocks_partitions_exactly():
+    for nb in (0, 1, 7, 131072, 3437):
+        for world in (1, 2, 3, 8):
+            seen = []
+            for r in range(world):
+                seen += list(dt8.shard_blocks(nb, r, world))
+            assert seen == list(range(nb))
+            sizes = [len(dt8.shard_blocks(nb, r, world)) for r in range(world)]
+            assert max(sizes) - min(sizes) <= 1
+    with pytest.raises(ValueError):
+        dt8.shard_blocks(10, 2, 2)

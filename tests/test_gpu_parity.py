@@ -1,0 +1,431 @@
+"""Parity of the CUDA library against the CPU checker, through the C ABI (via the thin binding).
+
+Same seeded inputs on both sides; integer results (codes) and absmax bit-exact, parameters within
+1e-6 relative (mixed with an rms floor), 100-step trajectories within 1e-4."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2412_01195_b200 as dt8
+from paper_2412_01195_b200 import synth
+from helpers import (AdamState, SgdState, assert_codes_match, assert_params_close, to_np,
+                     use_all_cores)
+
+pytestmark = pytest.mark.gpu
+F = np.float32
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _setup():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    dt8.dt8_init()
+    use_all_cores()
+    yield
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------------------------------------
+# quantize / dequantize
+# ------------------------------------------------------------------------------------------------
+def quant_roundtrip_check(x: torch.Tensor, B: int, signed: bool):
+    codes, absmax = dt8.dt8_quantize_blockwise(x.to(DEV), B, signed)
+    out = dt8.dt8_dequantize_blockwise(codes, absmax, B, signed)
+    torch.cuda.synchronize()
+    rc, ra = oracle.quantize_blockwise(to_np(x), B, signed)
+    assert np.array_equal(to_np(absmax), ra)
+    assert_codes_match(to_np(codes), rc)
+    assert np.array_equal(to_np(out), oracle.dequantize_blockwise(rc, ra, B, signed))
+
+
+@pytest.mark.parametrize("signed", [True, False])
+@pytest.mark.parametrize("B", [256, 512, 1024, 2048, 4096])
+def test_quantize_dequantize_sizes_and_tails(B, signed):
+    for n in (1, 3, 4, 5, B - 1, B, B + 1, 2 * B + 3, 37 * B + B // 2 + 1, 300 * B + 7):
+        x = synth.laplace_outliers(n, seed=300 + n % 97)
+        if not signed:
+            x = x.abs()
+        quant_roundtrip_check(x, B, signed)
+
+
+@pytest.mark.parametrize("signed", [True, False])
+def test_quantize_sweep_configuration(signed):
+    """Configuration 4 at its smaller sizes: Laplace(0,1) with 1e-3 outliers x100 (the 128M size is
+    covered by sampled blocks in the full-size test)."""
+    c = synth.QUANT_SWEEP
+    for n in c["sizes"][:2]:
+        x = synth.laplace_outliers(n, seed=c["seed"])
+        x = x if signed else x.abs()
+        for B in c["block_sizes"]:
+            quant_roundtrip_check(x, B, signed)
+
+
+def test_quantize_degenerate_blocks():
+    B = 256
+    x = torch.zeros(5 * B + 9)
+    x[B:2 * B] = synth.normal(B, 1e-30, 1)            # tiny maximum: division outside the fast range
+    x[2 * B:3 * B] = synth.normal(B, 1e30, 2)         # huge maximum
+    x[3 * B:4 * B] = synth.normal(B, 1e-42, 3)        # subnormal block
+    x[4 * B] = -7.0                                   # one non-zero element, negative
+    for signed in (True, False):
+        quant_roundtrip_check(x, B, signed)
+    codes, absmax = dt8.dt8_quantize_blockwise(torch.zeros(B, device=DEV), B, True)
+    assert torch.all(codes == 127) and torch.all(absmax == 0)
+    codes, absmax = dt8.dt8_quantize_blockwise(torch.zeros(0, device=DEV), B, True)
+    assert codes.numel() == 0 and absmax.numel() == 0
+    # unsigned table with negative inputs: they take the value 0
+    quant_roundtrip_check(synth.normal(3 * B + 1, 1.0, 4), B, False)
+
+
+@pytest.mark.parametrize("signed", [True, False])
+def test_quantize_follows_true_division(signed):
+    """Inputs on which x/N and x*(1/N) fall on different codes (Eq. quant1 divides)."""
+    Q = oracle.codebook(signed)
+    Q64 = Q.astype(np.float64)
+    mids = ((Q64[:-1] + Q64[1:]) / 2)[Q64[:-1] != Q64[1:]]
+    mids = mids[mids > 0].astype(F)
+    rng = np.random.default_rng(80)
+    B = 256
+    nblk = 4000
+    N = rng.uniform(0.5, 2.0, nblk).astype(F)
+    x = np.zeros((nblk, B), F)
+    x[:, 0] = N
+    T = rng.choice(mids, (nblk, B - 1))
+    x[:, 1:] = (T * N[:, None]).astype(F)             # x / N within an ulp of a mid-point
+    x[:, 1:] = np.minimum(np.abs(x[:, 1:]), N[:, None]) * (rng.choice([-1, 1], (nblk, B - 1)) if signed else 1)
+    quant_roundtrip_check(torch.from_numpy(x.ravel()), B, signed)
+
+
+@pytest.mark.parametrize("signed", [True, False])
+def test_encoder_over_a_strided_sweep_of_all_floats(signed):
+    """Blocks whose maximum is exactly 1, so the normalised value is the input itself: every 13th
+    binary32 bit pattern in [0, 1] (and its negative for the signed table)."""
+    Q = oracle.codebook(signed)
+    B = 256
+    bits = np.arange(0, 0x3F800000, 13, dtype=np.uint32)
+    bits = bits[: (bits.size // (B - 1)) * (B - 1)].reshape(-1, B - 1)
+    for sign in ((0, 0x80000000) if signed else (0,)):
+        x = np.empty((bits.shape[0], B), np.uint32)
+        x[:, 0] = 0x3F800000
+        x[:, 1:] = bits | np.uint32(sign)
+        xf = x.view(F).ravel()
+        codes, absmax = dt8.dt8_quantize_blockwise(torch.from_numpy(xf).to(DEV), B, signed)
+        torch.cuda.synchronize()
+        assert torch.all(absmax == 1.0)
+        assert_codes_match(to_np(codes), oracle.nearest(Q, xf))
+
+
+def test_dequantize_every_code_and_scale():
+    for signed in (True, False):
+        for N in (1.0, 3.7e-5, 2.0 ** -20, 1e4, 0.0):
+            codes = torch.arange(256, dtype=torch.uint8, device=DEV)
+            absmax = torch.tensor([N], dtype=torch.float32, device=DEV)
+            out = dt8.dt8_dequantize_blockwise(codes, absmax, 256, signed)
+            ref = oracle.dequantize_blockwise(np.arange(256, dtype=np.uint8), np.array([N], F), 256, signed)
+            assert np.array_equal(to_np(out).view(np.uint32), ref.view(np.uint32))
+
+
+# ------------------------------------------------------------------------------------------------
+# Adam
+# ------------------------------------------------------------------------------------------------
+def test_adam_configuration_1():
+    """1,048,576 elements, one AdamW step from the zero state (lr 1e-3, betas 0.9/0.999, wd 0)."""
+    c = synth.ADAM_FLAT_SMALL
+    w0, g = synth.flat_adam_inputs(c["n"], c["seed"])
+    st = AdamState(w0, c["block_size"])
+    st.step(g, 1, c)
+    st.check()
+    # closed form of the first step, straight from the inputs
+    g64 = g.numpy().astype(np.float64)
+    want = w0.numpy().astype(np.float64) - c["lr"] * g64 / (np.abs(g64) + c["eps"])
+    assert np.max(np.abs(to_np(st.w_gpu) - want)) <= 4e-7 * np.max(np.abs(want)) + 1e-10
+
+
+@pytest.mark.parametrize("B", [256, 512, 1024, 2048, 4096])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_adam_steps_all_block_sizes(B, gdtype):
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    for n in (1, B - 3, 5 * B + 11, 150 * B + B // 2):
+        st = AdamState(synth.normal(n, 0.02, 400 + B), B)
+        for t in range(1, 6):
+            st.step(synth.fresh_grad(n, 41, t, dtype=gdtype), t, hp)
+            st.check()
+
+
+def test_adam_trajectory_100_steps():
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    n, B = 200 * 2048 + 777, 2048
+    st = AdamState(synth.normal(n, 0.02, 500), B)
+    for t in range(1, 101):
+        st.step(synth.fresh_grad(n, 42, t), t, hp)
+        if t in (1, 2, 10, 50):
+            st.check()
+    st.check(rel=1e-4)
+    st.check(rel=1e-6)
+
+
+@pytest.mark.parametrize("flags", [0, dt8.DT8_ADAM_BIAS_CORRECTION, dt8.DT8_ADAM_DECOUPLED_WD])
+def test_adam_variants(flags):
+    """Literal Eq. adam (no bias correction), coupled L2 decay (IEEE parameter path: bit-exact)."""
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.05)
+    n, B = 33 * 2048 + 5, 2048
+    st = AdamState(synth.normal(n, 0.02, 600), B)
+    for t in range(1, 21):
+        st.step(synth.fresh_grad(n, 43, t), t, hp, flags)
+    st.check(exact_params=not (flags & dt8.DT8_ADAM_DECOUPLED_WD))
+
+
+def test_adam_heavy_tailed_and_sparse_gradients():
+    """Student-t gradients, zero gradients, and a block that stays all-zero."""
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    n, B = 20 * 2048, 2048
+    st = AdamState(synth.normal(n, 0.02, 700), B)
+    for t in range(1, 11):
+        g = synth.student_t(n, 3, 1e-3, 7100 + t)
+        g[3 * B:5 * B] = 0.0
+        g[7 * B:8 * B] *= 1e-20
+        g[9 * B + 5] = 50.0
+        st.step(g, t, hp)
+    st.check()
+    assert np.all(st.ma[3:5] == 0) and np.all(to_np(st.ma_gpu)[3:5] == 0)
+
+
+# ------------------------------------------------------------------------------------------------
+# SGD
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("B", [256, 512, 1024, 2048, 4096])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_sgd_steps_all_block_sizes(B, gdtype):
+    hp = dict(lr=0.1, momentum=0.9, weight_decay=1e-4)
+    for n in (2, B + 1, 7 * B + 13, 120 * B + 1):
+        st = SgdState(synth.normal(n, 0.05, 800 + B), B)
+        for t in range(1, 6):
+            g = synth.student_t(n, 3, 1e-3, 8100 + t)
+            st.step(g.to(gdtype), t, hp)
+            st.check()
+
+
+def test_sgd_configuration_2_multi_tensor_100_steps():
+    """37 conv3x3 weights (6,561,792 elements), Student-t gradients, momentum 0.9, wd 1e-4, lr 0.1,
+    100 steps; the list is stepped in one launch and must equal the checker tensor by tensor."""
+    c = synth.SGD_CONV
+    B = c["block_size"]
+    ws = synth.conv_sgd_params(c["seed"])
+    sizes = [w.numel() for w in ws]
+    assert sum(sizes) == 6_561_792 and len(sizes) == 37
+    w_gpu = [w.to(DEV) for w in ws]
+    st_gpu = [dt8.new_state(n, B, True, DEV) for n in sizes]
+    w_ref = [to_np(w) for w in ws]
+    mc_ref = [np.full(n, 127, np.uint8) for n in sizes]
+    ma_ref = [np.zeros(oracle.num_blocks(n, B), F) for n in sizes]
+    for t in range(1, c["steps"] + 1):
+        gs = synth.conv_sgd_grads(c["seed"], t)
+        dt8.dt8_sgd_step_multi(w_gpu, [g.to(DEV) for g in gs], [s[0] for s in st_gpu],
+                               [s[1] for s in st_gpu], c["lr"], c["momentum"], c["weight_decay"], t, B)
+        oracle.sgd_step_multi(w_ref, [to_np(g) for g in gs], mc_ref, ma_ref, c["lr"], c["momentum"],
+                              c["weight_decay"], t, B)
+        if t in (1, 2, 10, 100):
+            torch.cuda.synchronize()
+            for i in range(len(sizes)):
+                assert np.array_equal(to_np(st_gpu[i][1]), ma_ref[i])
+                assert_codes_match(to_np(st_gpu[i][0]), mc_ref[i])
+                assert np.array_equal(to_np(w_gpu[i]), w_ref[i])
+
+
+def test_adam_configuration_3_multi_tensor_100_steps():
+    """~200 tensors of a ResNet speaker extractor, bf16 gradients, AdamW wd 0.05, 100 steps."""
+    c = synth.ADAM_RESNET
+    B = c["block_size"]
+    ws = synth.resnet_adam_params(c["seed"])
+    sizes = [w.numel() for w in ws]
+    assert len(sizes) == 197 and 7.0e6 < sum(sizes) < 7.1e6 and min(sizes) == 32 and max(sizes) == 1_534_464
+    w_gpu = [w.to(DEV) for w in ws]
+    m_gpu = [dt8.new_state(n, B, True, DEV) for n in sizes]
+    r_gpu = [dt8.new_state(n, B, False, DEV) for n in sizes]
+    w_ref = [to_np(w) for w in ws]
+    mc = [np.full(n, 127, np.uint8) for n in sizes]
+    ma = [np.zeros(oracle.num_blocks(n, B), F) for n in sizes]
+    rc = [np.zeros(n, np.uint8) for n in sizes]
+    ra = [np.zeros(oracle.num_blocks(n, B), F) for n in sizes]
+    for t in range(1, c["steps"] + 1):
+        gs = synth.resnet_adam_grads(c["seed"], t)
+        dt8.dt8_adam_step_multi(w_gpu, [g.to(DEV) for g in gs], [s[0] for s in m_gpu], [s[1] for s in m_gpu],
+                                [s[0] for s in r_gpu], [s[1] for s in r_gpu], c["lr"], c["beta1"],
+                                c["beta2"], c["eps"], c["weight_decay"], t, B)
+        oracle.adam_step_multi(w_ref, [to_np(g) for g in gs], mc, ma, rc, ra, c["lr"], c["beta1"],
+                               c["beta2"], c["eps"], c["weight_decay"], t, B)
+        if t in (1, 3, 100):
+            torch.cuda.synchronize()
+            for i in range(len(sizes)):
+                assert np.array_equal(to_np(m_gpu[i][1]), ma[i]) and np.array_equal(to_np(r_gpu[i][1]), ra[i])
+                assert_codes_match(to_np(m_gpu[i][0]), mc[i])
+                assert_codes_match(to_np(r_gpu[i][0]), rc[i])
+                assert_params_close(to_np(w_gpu[i]), w_ref[i], 1e-4 if t == 100 else 1e-6)
+
+
+def test_multi_equals_single_and_skips_empty_tensors():
+    B = 512
+    sizes = [0, 5, B, 3 * B + 1, 0, 70 * B + 9]
+    hp = (1e-3, 0.9, 0.999, 1e-8, 0.01)
+    ws = [synth.normal(n, 0.02, 900 + i).to(DEV) for i, n in enumerate(sizes)]
+    gs = [synth.normal(n, 1e-3, 950 + i).to(DEV) for i, n in enumerate(sizes)]
+    a = [(w.clone(), *dt8.new_state(n, B, True, DEV), *dt8.new_state(n, B, False, DEV)) for w, n in zip(ws, sizes)]
+    b = [(w.clone(), *dt8.new_state(n, B, True, DEV), *dt8.new_state(n, B, False, DEV)) for w, n in zip(ws, sizes)]
+    for t in (1, 2, 3):
+        dt8.dt8_adam_step_multi([x[0] for x in a], gs, [x[1] for x in a], [x[2] for x in a],
+                                [x[3] for x in a], [x[4] for x in a], *hp, t, B)
+        for x, g in zip(b, gs):
+            dt8.dt8_adam_step(x[0], g, x[1], x[2], x[3], x[4], *hp, t, B)
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        for u, v in zip(x, y):
+            assert torch.equal(u, v)
+
+
+def test_more_tensors_than_one_launch_holds():
+    """600 small tensors: the pointer list is cut into several launches."""
+    B = 256
+    sizes = [17 + (i * 37) % 700 for i in range(600)]
+    ws = [synth.normal(n, 0.05, 1000 + i) for i, n in enumerate(sizes)]
+    gs = [synth.normal(n, 1e-3, 2000 + i) for i, n in enumerate(sizes)]
+    w_gpu = [w.to(DEV) for w in ws]
+    st = [dt8.new_state(n, B, True, DEV) for n in sizes]
+    dt8.dt8_sgd_step_multi(w_gpu, [g.to(DEV) for g in gs], [s[0] for s in st], [s[1] for s in st],
+                           0.1, 0.9, 1e-4, 1, B)
+    torch.cuda.synchronize()
+    for i, n in enumerate(sizes):
+        w, mc, ma = to_np(ws[i]), np.full(n, 127, np.uint8), np.zeros(oracle.num_blocks(n, B), F)
+        oracle.sgd_step(w, to_np(gs[i]), mc, ma, 0.1, 0.9, 1e-4, 1, B)
+        assert np.array_equal(to_np(w_gpu[i]), w) and np.array_equal(to_np(st[i][0]), mc)
+        assert np.array_equal(to_np(st[i][1]), ma)
+
+
+# ------------------------------------------------------------------------------------------------
+# memory safety, determinism, resume, streams
+# ------------------------------------------------------------------------------------------------
+def test_no_write_outside_the_buffers():
+    """Canary padding around every buffer, ragged sizes, checked after the kernels ran."""
+    B, pad = 1024, 64
+    for n in (1, B - 1, 3 * B + 2, 9 * B + 1023):
+        nb = dt8.num_blocks(n, B)
+
+        def padded(count, dtype, fill):
+            buf = torch.full((count + 2 * pad,), fill, dtype=dtype, device=DEV)
+            return buf, buf[pad:pad + count]
+
+        wbuf, w = padded(n, torch.float32, 777.0)
+        gbuf, g = padded(n, torch.float32, 777.0)
+        mcb, mc = padded(n, torch.uint8, 0xAB)
+        rcb, rc = padded(n, torch.uint8, 0xAB)
+        mab, ma = padded(nb, torch.float32, 777.0)
+        rab, ra = padded(nb, torch.float32, 777.0)
+        w.copy_(synth.normal(n, 0.02, 1).to(DEV)); g.copy_(synth.normal(n, 1e-3, 2).to(DEV))
+        mc.fill_(127); rc.zero_(); ma.zero_(); ra.zero_()
+        dt8.dt8_adam_step(w, g, mc, ma, rc, ra, 1e-3, 0.9, 0.999, 1e-8, 0.0, 1, B)
+        dt8.dt8_sgd_step(w, g, mc, ma, 0.1, 0.9, 0.0, 1, B)
+        dt8.dt8_quantize_blockwise(g, B, True, mc, ma)
+        dt8.dt8_dequantize_blockwise(mc, ma, B, True, w)
+        torch.cuda.synchronize()
+        for buf, fill in ((wbuf, 777.0), (gbuf, 777.0), (mab, 777.0), (rab, 777.0), (mcb, 0xAB), (rcb, 0xAB)):
+            assert torch.all(buf[:pad] == fill) and torch.all(buf[-pad:] == fill)
+
+
+def test_run_to_run_bit_reproducible_and_resume():
+    hp = (1e-3, 0.9, 0.999, 1e-8, 0.01)
+    n, B = 50 * 2048 + 3, 2048
+    w0 = synth.normal(n, 0.02, 1100).to(DEV)
+    grads = [synth.fresh_grad(n, 44, t).to(DEV) for t in range(1, 9)]
+
+    def run(snapshot_at=None, resume_from=None):
+        if resume_from is None:
+            state = [w0.clone(), *dt8.new_state(n, B, True, DEV), *dt8.new_state(n, B, False, DEV)]
+            start = 1
+        else:
+            state, start = [t.clone() for t in resume_from[0]], resume_from[1]
+        snap = None
+        for t in range(start, 9):
+            dt8.dt8_adam_step(state[0], grads[t - 1], *state[1:], *hp, t, B)
+            if t == snapshot_at:
+                snap = ([x.clone() for x in state], t + 1)
+        torch.cuda.synchronize()
+        return state, snap
+
+    a, snap = run(snapshot_at=4)
+    b, _ = run()
+    c, _ = run(resume_from=snap)
+    for x, y, z in zip(a, b, c):
+        assert torch.equal(x, y) and torch.equal(x, z)
+
+
+def test_side_stream():
+    n, B = 10 * 2048, 2048
+    s = torch.cuda.Stream()
+    w = synth.normal(n, 0.02, 1200).to(DEV)
+    g = synth.normal(n, 1e-3, 1201).to(DEV)
+    ref = AdamState(w.cpu(), B)
+    ref.step(g.cpu(), 1, dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0))
+    mc, ma = dt8.new_state(n, B, True, DEV)
+    rc, ra = dt8.new_state(n, B, False, DEV)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        dt8.dt8_adam_step(w, g, mc, ma, rc, ra, 1e-3, 0.9, 0.999, 1e-8, 0.0, 1, B)
+    s.synchronize()
+    assert torch.equal(mc, ref.mc_gpu) and torch.equal(ra, ref.ra_gpu) and torch.equal(w, ref.w_gpu)
+
+
+# ------------------------------------------------------------------------------------------------
+# full size, in the launch configuration the benchmark times
+# ------------------------------------------------------------------------------------------------
+def test_adam_configuration_5_full_size_sampled_blocks():
+    """2^28 elements, 10 warm-up AdamW steps + 1, wd 0.01.  Blocks are independent, so the checker
+    follows a fixed subset of blocks (first, last, every 64th) through all 11 steps."""
+    c = synth.ADAM_FLAT_LARGE
+    n, B = c["n"], c["block_size"]
+    nb = n // B
+    w, _ = synth.flat_adam_inputs(n, c["seed"], device=DEV)
+    mc, ma = dt8.new_state(n, B, True, DEV)
+    rc, ra = dt8.new_state(n, B, False, DEV)
+    blocks = torch.unique(torch.cat([torch.arange(0, nb, 64), torch.tensor([nb - 1])])).to(DEV)
+    idx = (blocks[:, None] * B + torch.arange(B, device=DEV)[None, :]).reshape(-1)
+    ns = idx.numel()
+    w_ref = to_np(w[idx])
+    mc_ref, ma_ref = np.full(ns, 127, np.uint8), np.zeros(ns // B, F)
+    rc_ref, ra_ref = np.zeros(ns, np.uint8), np.zeros(ns // B, F)
+    for t in range(1, c["prewarm_steps"] + 2):
+        g = synth.fresh_grad(n, c["seed"], t, device=DEV)
+        dt8.dt8_adam_step(w, g, mc, ma, rc, ra, c["lr"], c["beta1"], c["beta2"], c["eps"],
+                          c["weight_decay"], t, B)
+        oracle.adam_step(w_ref, to_np(g[idx]), mc_ref, ma_ref, rc_ref, ra_ref, c["lr"], c["beta1"],
+                         c["beta2"], c["eps"], c["weight_decay"], t, B)
+        del g
+    torch.cuda.synchronize()
+    assert np.array_equal(to_np(ma[blocks]), ma_ref) and np.array_equal(to_np(ra[blocks]), ra_ref)
+    assert_codes_match(to_np(mc[idx]), mc_ref)
+    assert_codes_match(to_np(rc[idx]), rc_ref)
+    assert_params_close(to_np(w[idx]), w_ref, 1e-6)
+    # properties that hold for every block at any size
+    assert torch.all(ma > 0) and torch.all(ra > 0)
+    assert int((mc.view(nb, B) == 255).any(1).logical_or((mc.view(nb, B) == 0).any(1)).sum()) == nb
+    assert int((rc.view(nb, B) == 255).any(1).sum()) == nb
+    assert not bool((mc == 128).any())
+
+
+def test_quantize_128m_sampled_blocks():
+    """Configuration 4 at 2^27 elements: checker on every 128th block."""
+    n = synth.QUANT_SWEEP["sizes"][2]
+    x = synth.laplace_outliers(n, seed=3, device=DEV)
+    for B in (256, 2048, 4096):
+        nb = n // B
+        blocks = torch.arange(0, nb, 128, device=DEV)
+        idx = (blocks[:, None] * B + torch.arange(B, device=DEV)[None, :]).reshape(-1)
+        for signed in (True, False):
+            xin = x if signed else x.abs()
+            codes, absmax = dt8.dt8_quantize_blockwise(xin, B, signed)
+            out = dt8.dt8_dequantize_blockwise(codes, absmax, B, signed)
+            rc, ra = oracle.quantize_blockwise(to_np(xin[idx]), B, signed)
+            assert np.array_equal(to_np(absmax[blocks]), ra)
+            assert_codes_match(to_np(codes[idx]), rc)
+            assert np.array_equal(to_np(out[idx]), oracle.dequantize_blockwise(rc, ra, B, signed))
+            assert torch.equal(absmax, xin.view(nb, B).abs().amax(1))
+            del codes, absmax, out

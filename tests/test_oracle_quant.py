@@ -184,3 +184,36 @@ def test_degenerate_inputs():
     assert codes.tolist() == [255, 0] and absmax.tolist() == [2.5, 2.5]
     with pytest.raises(ValueError):
         oracle.quantize_blockwise(np.zeros(4, np.float32), 0, True)
+
+
+def division_discriminators(signed, want=32, seed=16):
+    """Pairs (x, N) whose code differs between x / N (Eq. quant1 as written) and x * (1 / N)."""
+    Q = TABLES[signed]
+    Q64 = Q.astype(np.float64)
+    mids = ((Q64[:-1] + Q64[1:]) / 2)[Q64[:-1] != Q64[1:]]
+    mids = mids[mids > 0].astype(np.float32)
+    rng = np.random.default_rng(seed)
+    xs, Ns = [], []
+    while len(xs) < want:
+        N = rng.uniform(0.5, 2.0, 200000).astype(np.float32)
+        T = rng.choice(mids, N.size)
+        x = (T * N).astype(np.float32)                       # x / N lands within an ulp of a mid-point
+        v_div = x / N
+        v_rcp = x * (np.float32(1.0) / N)
+        differ = oracle.nearest(Q, v_div) != oracle.nearest(Q, v_rcp)
+        xs += x[differ].tolist()
+        Ns += N[differ].tolist()
+    return np.array(xs[:want], np.float32), np.array(Ns[:want], np.float32)
+
+
+@pytest.mark.parametrize("signed", [True, False])
+def test_normalisation_is_a_true_division(signed):
+    """Eq. quant1 divides by N_b.  Near a mid-point of the table a reciprocal-multiply lands on
+    the other code; on such inputs the block quantizer must follow the division."""
+    Q = TABLES[signed]
+    x, N = division_discriminators(signed)
+    for xi, Ni in zip(x, N):
+        codes, absmax = oracle.quantize_blockwise(np.array([xi, Ni], np.float32), 2, signed)
+        assert absmax[0] == Ni and codes[1] == 255
+        assert codes[0] == oracle.nearest(Q, np.array([xi / Ni], np.float32))[0]
+        assert codes[0] != oracle.nearest(Q, np.array([xi * (np.float32(1.0) / Ni)], np.float32))[0]
