@@ -68,10 +68,11 @@ int ensure_device(DeviceInfo* info, EncMeta* em) {
   return DT8_OK;
 }
 
-// Opt a kernel in to its dynamic shared memory size, once per device.
+// Opt a kernel in to its dynamic shared memory size, once per device.  `done` is the caller's
+// per-kernel flag word (kernels of different template arguments can share a pointer type, so the
+// flag cannot live in this function).
 template <class K>
-cudaError_t allow_smem(K kernel, int device, size_t bytes) {
-  static std::atomic<uint64_t> done{0};
+cudaError_t allow_smem(std::atomic<uint64_t>& done, K kernel, int device, size_t bytes) {
   const uint64_t bit = 1ull << device;
   if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -119,7 +120,8 @@ int launch_adam(const Args& args, int64_t blocks, const AdamHyper& h, const EncM
   constexpr int GROUPS = kCtaThreads / (B / VPT);
   auto kernel = adam_kernel<Args, B, VPT, GBF16, EXACT>;
   const size_t smem = smem_bytes(em, true, true, true, true);
-  cudaError_t e = allow_smem(kernel, di.device, smem);
+  static std::atomic<uint64_t> smem_ok{0};
+  cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
   if (e != cudaSuccess) return cuda_fail(e);
   kernel<<<grid_for(blocks, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(args, h, em);
   e = cudaGetLastError();
@@ -156,7 +158,8 @@ int launch_sgd(const Args& args, int64_t blocks, const SgdHyper& h, const EncMet
   constexpr int GROUPS = kCtaThreads / (B / VPT);
   auto kernel = sgd_kernel<Args, B, VPT, GBF16>;
   const size_t smem = smem_bytes(em, true, false, true, true);
-  cudaError_t e = allow_smem(kernel, di.device, smem);
+  static std::atomic<uint64_t> smem_ok{0};
+  cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
   if (e != cudaSuccess) return cuda_fail(e);
   kernel<<<grid_for(blocks, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(args, h, em);
   e = cudaGetLastError();
@@ -188,7 +191,8 @@ int launch_quantize(const float* x, int64_t n, uint8_t* codes, float* absmax, co
   constexpr int GROUPS = kCtaThreads / (B / VPT);
   auto kernel = quantize_kernel<B, VPT, SIGNED>;
   const size_t smem = smem_bytes(em, SIGNED, !SIGNED, false, true);
-  cudaError_t e = allow_smem(kernel, di.device, smem);
+  static std::atomic<uint64_t> smem_ok{0};
+  cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
   if (e != cudaSuccess) return cuda_fail(e);
   const int64_t nb = (n + B - 1) / B;
   kernel<<<grid_for(nb, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(x, codes, absmax, n, nb, em);
@@ -311,12 +315,14 @@ int dt8_dequantize_blockwise(const uint8_t* codes, const float* absmax, int64_t 
   cudaError_t e;
   if (is_signed) {
     const size_t smem = smem_bytes(em, true, false, true, false);
-    e = allow_smem(dequantize_kernel<true>, di.device, smem);
+    static std::atomic<uint64_t> smem_ok{0};
+    e = allow_smem(smem_ok, dequantize_kernel<true>, di.device, smem);
     if (e != cudaSuccess) return cuda_fail(e);
     dequantize_kernel<true><<<grid, kCtaThreads, smem, s>>>(codes, absmax, out, n, shift, em);
   } else {
     const size_t smem = smem_bytes(em, false, true, true, false);
-    e = allow_smem(dequantize_kernel<false>, di.device, smem);
+    static std::atomic<uint64_t> smem_ok{0};
+    e = allow_smem(smem_ok, dequantize_kernel<false>, di.device, smem);
     if (e != cudaSuccess) return cuda_fail(e);
     dequantize_kernel<false><<<grid, kCtaThreads, smem, s>>>(codes, absmax, out, n, shift, em);
   }
