@@ -254,11 +254,22 @@ int dt8_selfcheck_encode_host(int is_signed, const float* v_host, int64_t n, uin
   const Tables* ht = host_tables();
   if (!ht) return DT8_ERR_UNSUPPORTED;
   const EncTable& e = is_signed ? ht->enc_signed : ht->enc_unsigned;
-  for (int64_t i = 0; i < n; ++i) {
-    uint32_t bits;
-    std::memcpy(&bits, v_host + i, 4);
-    out_host[i] = static_cast<uint8_t>(is_signed ? encode_signed(e.entries, e.first_key, e.num_entries, bits)
-                                                 : encode_unsigned(e.entries, e.first_key, e.num_entries, bits));
+  const EncView view = make_view(e.entries, e.first_key, e.num_entries);
+  // groups of four, as the kernels do; the tail is padded with zeros
+  for (int64_t i = 0; i < n; i += 4) {
+    uint32_t bits[4] = {0, 0, 0, 0};
+    const int cnt = static_cast<int>(n - i < 4 ? n - i : 4);
+    std::memcpy(bits, v_host + i, 4 * static_cast<size_t>(cnt));
+    uint32_t packed;
+    if (is_signed) {
+      packed = finish_signed4(lookup_signed(view, bits[0]), lookup_signed(view, bits[1]),
+                              lookup_signed(view, bits[2]), lookup_signed(view, bits[3]), bits[0],
+                              bits[1], bits[2], bits[3]);
+    } else {
+      packed = finish_unsigned4(lookup_unsigned(view, bits[0]), lookup_unsigned(view, bits[1]),
+                                lookup_unsigned(view, bits[2]), lookup_unsigned(view, bits[3]));
+    }
+    for (int j = 0; j < cnt; ++j) out_host[i + j] = static_cast<uint8_t>(packed >> (8 * j));
   }
   return DT8_OK;
 }

@@ -27,12 +27,16 @@ namespace dt8 {
 
 constexpr int kSignedShift = 16;    // 7 mantissa bits per bucket: width <= 2^-7 of the value
 constexpr int kUnsignedShift = 15;  // 8 mantissa bits per bucket
-constexpr uint32_t kNoThreshold = 0x7FFFFFu;
 constexpr int kMaxEncEntries = 6656;
 
-// entry = count_below | tie_flag << 8 | threshold_low_bits << 9
+// Entry layouts (low byte = number of thresholds below the bucket, i.e. the magnitude pattern at
+// the bucket's lower edge; the bits between it and the threshold field are all ones so that the
+// compare below is decided by the threshold field alone):
+//   signed   : T2 << 15 | 0x7F00 | count,  T2 = 2*threshold_low16 + (tie flag ? 0 : 1), 17 bits
+//   unsigned : thr << 17 | 0x1FF00 | count, thr = threshold_low15
+// A bucket without a threshold stores the all-ones field, which no query exceeds.
 struct EncTable {
-  int shift;            // bucket = bits(a) >> shift
+  int shift;            // bucket key = bits(a) >> shift
   uint32_t first_key;   // bucket key of the first regular bucket
   int num_entries;      // entry 0: everything below; last entry: a >= 1
   uint32_t entries[kMaxEncEntries];
@@ -49,40 +53,92 @@ struct Tables {
 void build_codebook(bool is_signed, float out[256]);
 
 // Builds all tables; returns false if an internal consistency check fails (two thresholds in one
-// bucket, more than 23 low bits, table overflow).
+// bucket, table overflow).
 bool build_tables(Tables* t);
 
 // The process-wide tables, built on first use (thread-safe).  nullptr if the build failed.
 const Tables* host_tables();
 
-// Magnitude pattern of `a_bits` (bits of a non-negative binary32); tie_up = 1 sends exact ties to
-// the larger magnitude.
-DT8_HD uint32_t encode_magnitude(const uint32_t* entries, int shift, uint32_t first_key,
-                                 int num_entries, uint32_t a_bits, uint32_t tie_up) {
-  int idx = (int)(a_bits >> shift) - (int)first_key + 1;
-  idx = idx < 0 ? 0 : idx;
-  idx = idx > num_entries - 1 ? num_entries - 1 : idx;
-  const uint32_t e = entries[idx];
-  const uint32_t low = (a_bits & ((1u << shift) - 1u)) + ((e >> 8) & tie_up);
-  return (e & 0xFFu) + (low > (e >> 9) ? 1u : 0u);
+// Byte permute with the semantics of the PTX prmt.b32 default mode: output byte i is byte
+// (nibble_i & 7) of the pair {y, x}; if bit 3 of the nibble is set the byte's sign bit is
+// replicated instead.
+DT8_HD uint32_t byte_perm(uint32_t x, uint32_t y, uint32_t sel) {
+#if defined(__CUDA_ARCH__)
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(x), "r"(y), "r"(sel));
+  return d;
+#else
+  const uint64_t src = (static_cast<uint64_t>(y) << 32) | x;
+  uint32_t d = 0;
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t nib = (sel >> (4 * i)) & 0xFu;
+    uint32_t b = static_cast<uint32_t>(src >> (8 * (nib & 7u))) & 0xFFu;
+    if (nib & 8u) b = (b & 0x80u) ? 0xFFu : 0u;
+    d |= b << (8 * i);
+  }
+  return d;
+#endif
 }
 
-// Code (index into the ascending signed table) of a normalised value given as raw bits.
-DT8_HD uint32_t encode_signed(const uint32_t* entries, uint32_t first_key, int num_entries,
-                              uint32_t v_bits) {
-  const uint32_t neg = v_bits >> 31;
-  const uint32_t p = encode_magnitude(entries, kSignedShift, first_key, num_entries,
-                                      v_bits & 0x7FFFFFFFu, neg);
-  const uint32_t c = neg ? 127u - p : 128u + p;
-  return p == 0u ? 127u : c;   // both zeros are stored as the first one
+// `biased` points (first_key - 1) entries before the table, so that the clamped bucket key
+// indexes it directly; lo_key = first_key - 1, hi_key = lo_key + num_entries - 1.
+struct EncView {
+  const uint32_t* biased;
+  uint32_t lo_key, hi_key;
+};
+
+DT8_HD EncView make_view(const uint32_t* entries, uint32_t first_key, int num_entries) {
+  EncView v;
+  v.lo_key = first_key - 1u;
+  v.hi_key = v.lo_key + static_cast<uint32_t>(num_entries) - 1u;
+  v.biased = entries - v.lo_key;
+  return v;
 }
 
-// Code of a normalised value for the unsigned table; negative values map to the value 0.
-DT8_HD uint32_t encode_unsigned(const uint32_t* entries, uint32_t first_key, int num_entries,
-                                uint32_t v_bits) {
-  const int32_t s = (int32_t)v_bits;
-  const uint32_t a_bits = s < 0 ? 0u : (uint32_t)s;
-  return encode_magnitude(entries, kUnsignedShift, first_key, num_entries, a_bits, 0u);
+// Signed table.  Returns a word whose low byte is the magnitude pattern p of |v| (exact ties go
+// down for v > 0 and up for v < 0, i.e. to the lower index of the ascending table).
+// x = v rotated by 16 bits: [mantissa_low16 | sign | exponent+mantissa_high7]; its top 17 bits are
+// 2*low16 + sign, which is compared with T2; its low 15 bits are the bucket key.
+DT8_HD uint32_t lookup_signed(const EncView& t, uint32_t v_bits) {
+  const uint32_t x = byte_perm(v_bits, 0u, 0x1032u);
+  uint32_t key = x & 0x7FFFu;
+  key = key < t.lo_key ? t.lo_key : key;
+  key = key > t.hi_key ? t.hi_key : key;
+  const uint32_t e = t.biased[key];
+  return e + (x > e ? 1u : 0u);
+}
+
+// Unsigned table; negative values (and -0) count as 0.
+DT8_HD uint32_t lookup_unsigned(const EncView& t, uint32_t v_bits) {
+  const int32_t lo_bits = static_cast<int32_t>(t.lo_key << kUnsignedShift);
+  int32_t s = static_cast<int32_t>(v_bits);
+  s = s < lo_bits ? lo_bits : s;                      // also maps negatives to the lowest bucket
+  const uint32_t a = static_cast<uint32_t>(s);
+  uint32_t key = a >> kUnsignedShift;
+  key = key > t.hi_key ? t.hi_key : key;
+  const uint32_t e = t.biased[key];
+  return e + ((a << (32 - kUnsignedShift)) > e ? 1u : 0u);
+}
+
+// Gathers the low bytes of four words into one word (word 0 in byte 0).
+DT8_HD uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  return byte_perm(byte_perm(a, b, 0x0040u), byte_perm(c, d, 0x0040u), 0x5410u);
+}
+
+// Four signed codes from four looked-up words and the four normalised values they came from:
+// code = 128 + p for v > 0, 127 - p for v < 0, and 127 whenever p == 0 (both zeros of the table
+// are stored as the first one).  127 - p == p ^ 0x7F and 128 + p == p ^ 0x80 for p <= 127.
+DT8_HD uint32_t finish_signed4(uint32_t e0, uint32_t e1, uint32_t e2, uint32_t e3, uint32_t v0,
+                               uint32_t v1, uint32_t v2, uint32_t v3) {
+  const uint32_t P = pack_low_bytes(e0, e1, e2, e3);
+  const uint32_t top = byte_perm(byte_perm(v0, v1, 0x0073u), byte_perm(v2, v3, 0x0073u), 0x5410u);
+  const uint32_t nonzero = P + 0x7F7F7F7Fu;                 // bit 7 of a byte set iff p >= 1
+  const uint32_t flip = byte_perm(top | ~nonzero, 0u, 0xBA98u);  // 0xFF where v < 0 or p == 0
+  return P ^ 0x80808080u ^ flip;
+}
+
+DT8_HD uint32_t finish_unsigned4(uint32_t e0, uint32_t e1, uint32_t e2, uint32_t e3) {
+  return pack_low_bytes(e0, e1, e2, e3);
 }
 
 }  // namespace dt8
