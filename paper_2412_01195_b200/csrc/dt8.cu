@@ -96,9 +96,34 @@ int grid_for(int64_t blocks, int groups_per_cta, int sm_count) {
   return static_cast<int>(want < sm_count ? want : sm_count);
 }
 
-// Values per thread for each supported block size.
-template <int B> struct Geometry { static constexpr int VPT = 8; };
-
+// Values per thread and threads per CTA for each operation and block size.  A group (B / VPT
+// threads) is at least one warp, and the groups tile the CTA.
+#ifndef DT8_ADAM_VPT
+#define DT8_ADAM_VPT 16
+#endif
+#ifndef DT8_ADAM_THREADS
+#define DT8_ADAM_THREADS 512
+#endif
+#ifndef DT8_SGD_VPT
+#define DT8_SGD_VPT 16
+#endif
+#ifndef DT8_SGD_THREADS
+#define DT8_SGD_THREADS 512
+#endif
+#ifndef DT8_QUANT_VPT
+#define DT8_QUANT_VPT 8
+#endif
+#ifndef DT8_QUANT_THREADS
+#define DT8_QUANT_THREADS 1024
+#endif
+template <int B, int VPT_WANTED, int THREADS_WANTED> struct GeometryOf {
+  static constexpr int VPT = (B / VPT_WANTED >= 32) ? VPT_WANTED : B / 32;
+  static constexpr int THREADS = (THREADS_WANTED % (B / VPT) == 0) ? THREADS_WANTED : (B / VPT);
+  static_assert(VPT % 4 == 0 && THREADS <= kCtaThreads && THREADS % (B / VPT) == 0, "bad geometry");
+};
+template <int B> using AdamGeometry = GeometryOf<B, DT8_ADAM_VPT, DT8_ADAM_THREADS>;
+template <int B> using SgdGeometry = GeometryOf<B, DT8_SGD_VPT, DT8_SGD_THREADS>;
+template <int B> using QuantGeometry = GeometryOf<B, DT8_QUANT_VPT, DT8_QUANT_THREADS>;
 
 int check_tensor(const TensorDesc& d, int g_dtype, bool adam) {
   if (d.n < 0) return DT8_ERR_INVALID_ARG;
@@ -113,40 +138,47 @@ int check_tensor(const TensorDesc& d, int g_dtype, bool adam) {
 }
 
 // ---- launchers -------------------------------------------------------------------------------
-template <class Args, int B, bool GBF16, bool EXACT>
+template <class Args, int B, bool GBF16, int MODE>
 int launch_adam(const Args& args, int64_t blocks, const AdamHyper& h, const EncMeta& em,
                 const DeviceInfo& di, cudaStream_t stream) {
-  constexpr int VPT = Geometry<B>::VPT;
-  constexpr int GROUPS = kCtaThreads / (B / VPT);
-  auto kernel = adam_kernel<Args, B, VPT, GBF16, EXACT>;
+  constexpr int VPT = AdamGeometry<B>::VPT, THREADS = AdamGeometry<B>::THREADS;
+  constexpr int GROUPS = THREADS / (B / VPT);
+  auto kernel = block_kernel<AdamOp<B, VPT, THREADS, GBF16, MODE>, Args>;
   const size_t smem = smem_bytes(em, true, true, true, true);
   static std::atomic<uint64_t> smem_ok{0};
   cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
   if (e != cudaSuccess) return cuda_fail(e);
-  kernel<<<grid_for(blocks, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(args, h, em);
+  kernel<<<grid_for(blocks, GROUPS, di.sm_count), THREADS, smem, stream>>>(args, h, em);
   e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
 
+template <class Args, int B, bool GBF16>
+int dispatch_adam_mode(const Args& args, int64_t blocks, int mode, const AdamHyper& h,
+                       const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
+  switch (mode) {
+    case kAdamWFast: return launch_adam<Args, B, GBF16, kAdamWFast>(args, blocks, h, em, di, s);
+    case kAdamWIeee: return launch_adam<Args, B, GBF16, kAdamWIeee>(args, blocks, h, em, di, s);
+    default: return launch_adam<Args, B, GBF16, kAdamL2>(args, blocks, h, em, di, s);
+  }
+}
+
 template <class Args, int B>
-int dispatch_adam(const Args& args, int64_t blocks, int g_dtype, bool exact, const AdamHyper& h,
+int dispatch_adam(const Args& args, int64_t blocks, int g_dtype, int mode, const AdamHyper& h,
                   const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
-  if (g_dtype == DT8_BF16)
-    return exact ? launch_adam<Args, B, true, true>(args, blocks, h, em, di, s)
-                 : launch_adam<Args, B, true, false>(args, blocks, h, em, di, s);
-  return exact ? launch_adam<Args, B, false, true>(args, blocks, h, em, di, s)
-               : launch_adam<Args, B, false, false>(args, blocks, h, em, di, s);
+  return g_dtype == DT8_BF16 ? dispatch_adam_mode<Args, B, true>(args, blocks, mode, h, em, di, s)
+                             : dispatch_adam_mode<Args, B, false>(args, blocks, mode, h, em, di, s);
 }
 
 template <class Args>
-int dispatch_adam_b(const Args& args, int64_t blocks, int B, int g_dtype, bool exact,
+int dispatch_adam_b(const Args& args, int64_t blocks, int B, int g_dtype, int mode,
                     const AdamHyper& h, const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
   switch (B) {
-    case 256: return dispatch_adam<Args, 256>(args, blocks, g_dtype, exact, h, em, di, s);
-    case 512: return dispatch_adam<Args, 512>(args, blocks, g_dtype, exact, h, em, di, s);
-    case 1024: return dispatch_adam<Args, 1024>(args, blocks, g_dtype, exact, h, em, di, s);
-    case 2048: return dispatch_adam<Args, 2048>(args, blocks, g_dtype, exact, h, em, di, s);
-    case 4096: return dispatch_adam<Args, 4096>(args, blocks, g_dtype, exact, h, em, di, s);
+    case 256: return dispatch_adam<Args, 256>(args, blocks, g_dtype, mode, h, em, di, s);
+    case 512: return dispatch_adam<Args, 512>(args, blocks, g_dtype, mode, h, em, di, s);
+    case 1024: return dispatch_adam<Args, 1024>(args, blocks, g_dtype, mode, h, em, di, s);
+    case 2048: return dispatch_adam<Args, 2048>(args, blocks, g_dtype, mode, h, em, di, s);
+    case 4096: return dispatch_adam<Args, 4096>(args, blocks, g_dtype, mode, h, em, di, s);
   }
   return DT8_ERR_UNSUPPORTED;
 }
@@ -154,14 +186,14 @@ int dispatch_adam_b(const Args& args, int64_t blocks, int B, int g_dtype, bool e
 template <class Args, int B, bool GBF16>
 int launch_sgd(const Args& args, int64_t blocks, const SgdHyper& h, const EncMeta& em,
                const DeviceInfo& di, cudaStream_t stream) {
-  constexpr int VPT = Geometry<B>::VPT;
-  constexpr int GROUPS = kCtaThreads / (B / VPT);
-  auto kernel = sgd_kernel<Args, B, VPT, GBF16>;
+  constexpr int VPT = SgdGeometry<B>::VPT, THREADS = SgdGeometry<B>::THREADS;
+  constexpr int GROUPS = THREADS / (B / VPT);
+  auto kernel = block_kernel<SgdOp<B, VPT, THREADS, GBF16>, Args>;
   const size_t smem = smem_bytes(em, true, false, true, true);
   static std::atomic<uint64_t> smem_ok{0};
   cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
   if (e != cudaSuccess) return cuda_fail(e);
-  kernel<<<grid_for(blocks, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(args, h, em);
+  kernel<<<grid_for(blocks, GROUPS, di.sm_count), THREADS, smem, stream>>>(args, h, em);
   e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
@@ -187,15 +219,17 @@ int dispatch_sgd_b(const Args& args, int64_t blocks, int B, int g_dtype, const S
 template <int B, bool SIGNED>
 int launch_quantize(const float* x, int64_t n, uint8_t* codes, float* absmax, const EncMeta& em,
                     const DeviceInfo& di, cudaStream_t stream) {
-  constexpr int VPT = Geometry<B>::VPT;
-  constexpr int GROUPS = kCtaThreads / (B / VPT);
-  auto kernel = quantize_kernel<B, VPT, SIGNED>;
+  constexpr int VPT = QuantGeometry<B>::VPT, THREADS = QuantGeometry<B>::THREADS;
+  constexpr int GROUPS = THREADS / (B / VPT);
+  auto kernel = block_kernel<QuantOp<B, VPT, THREADS, SIGNED>, SingleArgs>;
   const size_t smem = smem_bytes(em, SIGNED, !SIGNED, false, true);
   static std::atomic<uint64_t> smem_ok{0};
   cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
   if (e != cudaSuccess) return cuda_fail(e);
-  const int64_t nb = (n + B - 1) / B;
-  kernel<<<grid_for(nb, GROUPS, di.sm_count), kCtaThreads, smem, stream>>>(x, codes, absmax, n, nb, em);
+  SingleArgs a;
+  a.t = TensorDesc{nullptr, x, codes, absmax, nullptr, nullptr, n};
+  a.nb = (n + B - 1) / B;
+  kernel<<<grid_for(a.nb, GROUPS, di.sm_count), THREADS, smem, stream>>>(a, NoHyper{0}, em);
   e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
@@ -221,6 +255,15 @@ AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float w
   h.step_scale = lr / h.bc1;
   h.ibc2 = 1.0f / h.bc2;
   return h;
+}
+
+// The single-instruction root and reciprocal flush subnormal numbers to zero; a flushed root
+// (below 1.1e-19) is invisible next to eps only while eps is well above it.
+constexpr float kMinEpsForFastUpdate = 1e-12f;
+
+int adam_mode(uint32_t flags, float eps) {
+  if (!(flags & DT8_ADAM_DECOUPLED_WD)) return kAdamL2;
+  return eps >= kMinEpsForFastUpdate ? kAdamWFast : kAdamWIeee;
 }
 
 }  // namespace
@@ -320,8 +363,9 @@ int dt8_dequantize_blockwise(const uint8_t* codes, const float* absmax, int64_t 
   if (rc != DT8_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t quads = (n + 3) / 4;
-  const int64_t ctas = (quads + kCtaThreads - 1) / kCtaThreads;
-  const int grid = static_cast<int>(ctas < 2 * di.sm_count ? ctas : 2 * di.sm_count);
+  const int64_t per_cta = static_cast<int64_t>(kCtaThreads) * kDeqUnroll;
+  const int64_t ctas = (quads + per_cta - 1) / per_cta;
+  const int grid = static_cast<int>(ctas < di.sm_count ? ctas : di.sm_count);
   const int shift = log2_int(block_size);
   cudaError_t e;
   if (is_signed) {
@@ -377,8 +421,7 @@ int dt8_adam_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float*
   rc = ensure_device(&di, &em);
   if (rc != DT8_OK) return rc;
   const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
-  const bool exact = !(flags & DT8_ADAM_DECOUPLED_WD);
-  return dispatch_adam_b(a, a.nb, block_size, g_dtype, exact, h, em, di,
+  return dispatch_adam_b(a, a.nb, block_size, g_dtype, adam_mode(flags, eps), h, em, di,
                          static_cast<cudaStream_t>(stream));
 }
 
@@ -461,11 +504,11 @@ int dt8_adam_step_multi(int num_tensors, float* const* p, const void* const* g, 
                         void* stream) {
   if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
   const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
-  const bool exact = !(flags & DT8_ADAM_DECOUPLED_WD);
+  const int mode = adam_mode(flags, eps);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   return run_multi(num_tensors, p, g, g_dtype, m_codes, m_absmax, r_codes, r_absmax, n, block_size,
                    true, [&](const MultiArgs& a, int64_t blocks, const EncMeta& em, const DeviceInfo& di) {
-                     return dispatch_adam_b(a, blocks, block_size, g_dtype, exact, h, em, di, s);
+                     return dispatch_adam_b(a, blocks, block_size, g_dtype, mode, h, em, di, s);
                    });
 }
 

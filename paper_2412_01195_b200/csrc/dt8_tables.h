@@ -99,23 +99,26 @@ DT8_HD EncView make_view(const uint32_t* entries, uint32_t first_key, int num_en
 // down for v > 0 and up for v < 0, i.e. to the lower index of the ascending table).
 // x = v rotated by 16 bits: [mantissa_low16 | sign | exponent+mantissa_high7]; its top 17 bits are
 // 2*low16 + sign, which is compared with T2; its low 15 bits are the bucket key.
+// CLAMP_HI = false may be used only when |v| <= 1 is known (the key then never exceeds hi_key).
+template <bool CLAMP_HI = true>
 DT8_HD uint32_t lookup_signed(const EncView& t, uint32_t v_bits) {
   const uint32_t x = byte_perm(v_bits, 0u, 0x1032u);
   uint32_t key = x & 0x7FFFu;
   key = key < t.lo_key ? t.lo_key : key;
-  key = key > t.hi_key ? t.hi_key : key;
+  if (CLAMP_HI) key = key > t.hi_key ? t.hi_key : key;
   const uint32_t e = t.biased[key];
   return e + (x > e ? 1u : 0u);
 }
 
 // Unsigned table; negative values (and -0) count as 0.
+template <bool CLAMP_HI = true>
 DT8_HD uint32_t lookup_unsigned(const EncView& t, uint32_t v_bits) {
   const int32_t lo_bits = static_cast<int32_t>(t.lo_key << kUnsignedShift);
   int32_t s = static_cast<int32_t>(v_bits);
   s = s < lo_bits ? lo_bits : s;                      // also maps negatives to the lowest bucket
   const uint32_t a = static_cast<uint32_t>(s);
   uint32_t key = a >> kUnsignedShift;
-  key = key > t.hi_key ? t.hi_key : key;
+  if (CLAMP_HI) key = key > t.hi_key ? t.hi_key : key;
   const uint32_t e = t.biased[key];
   return e + ((a << (32 - kUnsignedShift)) > e ? 1u : 0u);
 }
