@@ -111,7 +111,7 @@ int grid_for(int64_t blocks, int groups_per_cta, int sm_count) {
 #define DT8_SGD_THREADS 512
 #endif
 #ifndef DT8_QUANT_VPT
-#define DT8_QUANT_VPT 8
+#define DT8_QUANT_VPT 16
 #endif
 #ifndef DT8_QUANT_THREADS
 #define DT8_QUANT_THREADS 1024
