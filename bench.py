@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 
 METRIC = "adam8bit_step_effective_hbm_bandwidth"
 UNIT = "GB/s"
-WORKLOAD = "adam8bit_flat_2^28_fp32grad_block2048_wd0.01_prewarm10 (BASELINE configs[4])"
+WORKLOAD = "adam8bit_flat_2^28_fp32grad_block2048_wd0.01_prewarm10"
 DATASHEET_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
 
@@ -229,7 +229,7 @@ def run_dt8(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": round(gbs_per_gpu, 2), "peak": peak, "unit": "GB/s",
                      "frac": round(gbs_per_gpu / peak, 4), "traffic": args.traffic_bytes,
-                     "kernel": "dt8::adam_kernel<SingleArgs,2048,8,false,false>",
+                     "kernel": "dt8::block_kernel<AdamOp<2048,16,512,f32 grads,AdamW>,SingleArgs>",
                      "algorithmic_bytes_per_launch": bytes_step, "peak_source": peak_src,
                      "per_launch_ms": round(ms_step, 5)},
     }

@@ -52,6 +52,24 @@ int ensure_device(DeviceInfo* info, EncMeta* em) {
       std::memcpy(staging.enc_u, ht->enc_unsigned.entries, sizeof(uint32_t) * ht->enc_unsigned.num_entries);
       e = cudaMemcpyToSymbol(g_tables, &staging, sizeof(staging));
       if (e != cudaSuccess) return cuda_fail(e);
+      // The kernels address their shared-memory tables absolutely: check once that this build's
+      // tables fit the layout and that dynamic shared memory starts low enough on this device.
+      EncMeta probe_em;
+      probe_em.s_first = ht->enc_signed.first_key;
+      probe_em.u_first = ht->enc_unsigned.first_key;
+      probe_em.s_n = ht->enc_signed.num_entries;
+      probe_em.u_n = ht->enc_unsigned.num_entries;
+      if (!layout_ok(probe_em)) return DT8_ERR_UNSUPPORTED;
+      const int probe_smem = static_cast<int>(smem_bytes(probe_em, true, true, true, true));
+      e = cudaFuncSetAttribute(smem_start_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem);
+      if (e != cudaSuccess) return cuda_fail(e);
+      smem_start_probe<<<1, 32, probe_smem>>>();
+      e = cudaGetLastError();
+      if (e != cudaSuccess) return cuda_fail(e);
+      uint32_t smem_start = 0xFFFFFFFFu;
+      e = cudaMemcpyFromSymbol(&smem_start, g_smem_start, sizeof(smem_start));
+      if (e != cudaSuccess) return cuda_fail(e);
+      if (smem_start > kMaxSmemStart) return DT8_ERR_UNSUPPORTED;
       int sms = 0;
       e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
       if (e != cudaSuccess) return cuda_fail(e);
@@ -252,18 +270,19 @@ AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float w
     h.bc1 = 1.0f;
     h.bc2 = 1.0f;
   }
-  h.step_scale = lr / h.bc1;
-  h.ibc2 = 1.0f / h.bc2;
+  const double root_bc2 = std::sqrt(static_cast<double>(h.bc2));
+  h.step_scale = static_cast<float>(static_cast<double>(lr) * root_bc2 / static_cast<double>(h.bc1));
+  h.eps_scaled = static_cast<float>(static_cast<double>(eps) * root_bc2);
   return h;
 }
 
 // The single-instruction root and reciprocal flush subnormal numbers to zero; a flushed root
-// (below 1.1e-19) is invisible next to eps only while eps is well above it.
+// (below 1.1e-19) is invisible next to the scaled eps only while that is well above it.
 constexpr float kMinEpsForFastUpdate = 1e-12f;
 
-int adam_mode(uint32_t flags, float eps) {
+int adam_mode(uint32_t flags, const AdamHyper& h) {
   if (!(flags & DT8_ADAM_DECOUPLED_WD)) return kAdamL2;
-  return eps >= kMinEpsForFastUpdate ? kAdamWFast : kAdamWIeee;
+  return h.eps_scaled >= kMinEpsForFastUpdate ? kAdamWFast : kAdamWIeee;
 }
 
 }  // namespace
@@ -297,7 +316,8 @@ int dt8_selfcheck_encode_host(int is_signed, const float* v_host, int64_t n, uin
   const Tables* ht = host_tables();
   if (!ht) return DT8_ERR_UNSUPPORTED;
   const EncTable& e = is_signed ? ht->enc_signed : ht->enc_unsigned;
-  const EncView view = make_view(e.entries, e.first_key, e.num_entries);
+  const EncBounds bounds = make_bounds(e.first_key, e.num_entries);
+  const HostFetch fetch{e.entries, bounds.lo4};
   // groups of four, as the kernels do; the tail is padded with zeros
   for (int64_t i = 0; i < n; i += 4) {
     uint32_t bits[4] = {0, 0, 0, 0};
@@ -305,12 +325,16 @@ int dt8_selfcheck_encode_host(int is_signed, const float* v_host, int64_t n, uin
     std::memcpy(bits, v_host + i, 4 * static_cast<size_t>(cnt));
     uint32_t packed;
     if (is_signed) {
-      packed = finish_signed4(lookup_signed(view, bits[0]), lookup_signed(view, bits[1]),
-                              lookup_signed(view, bits[2]), lookup_signed(view, bits[3]), bits[0],
-                              bits[1], bits[2], bits[3]);
+      packed = finish_signed4(lookup_signed<true>(fetch, bounds, bits[0]),
+                              lookup_signed<true>(fetch, bounds, bits[1]),
+                              lookup_signed<true>(fetch, bounds, bits[2]),
+                              lookup_signed<true>(fetch, bounds, bits[3]), bits[0], bits[1], bits[2],
+                              bits[3]);
     } else {
-      packed = finish_unsigned4(lookup_unsigned(view, bits[0]), lookup_unsigned(view, bits[1]),
-                                lookup_unsigned(view, bits[2]), lookup_unsigned(view, bits[3]));
+      packed = finish_unsigned4(lookup_unsigned<true>(fetch, bounds, bits[0]),
+                                lookup_unsigned<true>(fetch, bounds, bits[1]),
+                                lookup_unsigned<true>(fetch, bounds, bits[2]),
+                                lookup_unsigned<true>(fetch, bounds, bits[3]));
     }
     for (int j = 0; j < cnt; ++j) out_host[i + j] = static_cast<uint8_t>(packed >> (8 * j));
   }
@@ -421,7 +445,7 @@ int dt8_adam_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float*
   rc = ensure_device(&di, &em);
   if (rc != DT8_OK) return rc;
   const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
-  return dispatch_adam_b(a, a.nb, block_size, g_dtype, adam_mode(flags, eps), h, em, di,
+  return dispatch_adam_b(a, a.nb, block_size, g_dtype, adam_mode(flags, h), h, em, di,
                          static_cast<cudaStream_t>(stream));
 }
 
@@ -504,7 +528,7 @@ int dt8_adam_step_multi(int num_tensors, float* const* p, const void* const* g, 
                         void* stream) {
   if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
   const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
-  const int mode = adam_mode(flags, eps);
+  const int mode = adam_mode(flags, h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   return run_multi(num_tensors, p, g, g_dtype, m_codes, m_absmax, r_codes, r_absmax, n, block_size,
                    true, [&](const MultiArgs& a, int64_t blocks, const EncMeta& em, const DeviceInfo& di) {

@@ -80,47 +80,55 @@ DT8_HD uint32_t byte_perm(uint32_t x, uint32_t y, uint32_t sel) {
 #endif
 }
 
-// `biased` points (first_key - 1) entries before the table, so that the clamped bucket key
-// indexes it directly; lo_key = first_key - 1, hi_key = lo_key + num_entries - 1.
-struct EncView {
-  const uint32_t* biased;
-  uint32_t lo_key, hi_key;
+// Bounds of one encode table in "byte address" form: bucket key k is looked up at byte offset
+// 4*k.  lo4 = 4*(first_key - 1) is the entry "everything below", hi4 the entry "a >= 1".  In the
+// kernels the table is placed in shared memory so that 4*k IS the shared-memory address of the
+// entry of key k (no base to add); on the host HostFetch maps the offset back to the array.
+struct EncBounds {
+  uint32_t lo4, hi4;
 };
 
-DT8_HD EncView make_view(const uint32_t* entries, uint32_t first_key, int num_entries) {
-  EncView v;
-  v.lo_key = first_key - 1u;
-  v.hi_key = v.lo_key + static_cast<uint32_t>(num_entries) - 1u;
-  v.biased = entries - v.lo_key;
-  return v;
+DT8_HD EncBounds make_bounds(uint32_t first_key, int num_entries) {
+  EncBounds b;
+  b.lo4 = 4u * (first_key - 1u);
+  b.hi4 = b.lo4 + 4u * (static_cast<uint32_t>(num_entries) - 1u);
+  return b;
 }
+
+struct HostFetch {
+  const uint32_t* entries;
+  uint32_t lo4;
+  DT8_HD uint32_t operator()(uint32_t k4) const { return entries[(k4 - lo4) >> 2]; }
+};
 
 // Signed table.  Returns a word whose low byte is the magnitude pattern p of |v| (exact ties go
 // down for v > 0 and up for v < 0, i.e. to the lower index of the ascending table).
 // x = v rotated by 16 bits: [mantissa_low16 | sign | exponent+mantissa_high7]; its top 17 bits are
 // 2*low16 + sign, which is compared with T2; its low 15 bits are the bucket key.
-// CLAMP_HI = false may be used only when |v| <= 1 is known (the key then never exceeds hi_key).
-template <bool CLAMP_HI = true>
-DT8_HD uint32_t lookup_signed(const EncView& t, uint32_t v_bits) {
+// CLAMP_HI = false may be used only when |v| <= 1 is known (the key then never exceeds hi4).
+template <bool CLAMP_HI, class Fetch>
+DT8_HD uint32_t lookup_signed(const Fetch& fetch, const EncBounds& t, uint32_t v_bits) {
   const uint32_t x = byte_perm(v_bits, 0u, 0x1032u);
-  uint32_t key = x & 0x7FFFu;
-  key = key < t.lo_key ? t.lo_key : key;
-  if (CLAMP_HI) key = key > t.hi_key ? t.hi_key : key;
-  const uint32_t e = t.biased[key];
+  uint32_t k4 = (x << 2) & 0x1FFFCu;
+  k4 = k4 < t.lo4 ? t.lo4 : k4;
+  if (CLAMP_HI) k4 = k4 > t.hi4 ? t.hi4 : k4;
+  const uint32_t e = fetch(k4);
   return e + (x > e ? 1u : 0u);
 }
 
-// Unsigned table; negative values (and -0) count as 0.
-template <bool CLAMP_HI = true>
-DT8_HD uint32_t lookup_unsigned(const EncView& t, uint32_t v_bits) {
-  const int32_t lo_bits = static_cast<int32_t>(t.lo_key << kUnsignedShift);
+// Unsigned table; negative values (and -0) count as 0.  lo4 << 13 is the bit pattern of the
+// lower edge of the lowest bucket (4 * key << 13 == key << kUnsignedShift).
+template <bool CLAMP_HI, class Fetch>
+DT8_HD uint32_t lookup_unsigned(const Fetch& fetch, const EncBounds& t, uint32_t v_bits) {
+  static_assert(kUnsignedShift == 15, "offset arithmetic below assumes a 15-bit bucket");
+  const int32_t lo_bits = static_cast<int32_t>(t.lo4 << 13);
   int32_t s = static_cast<int32_t>(v_bits);
   s = s < lo_bits ? lo_bits : s;                      // also maps negatives to the lowest bucket
   const uint32_t a = static_cast<uint32_t>(s);
-  uint32_t key = a >> kUnsignedShift;
-  if (CLAMP_HI) key = key > t.hi_key ? t.hi_key : key;
-  const uint32_t e = t.biased[key];
-  return e + ((a << (32 - kUnsignedShift)) > e ? 1u : 0u);
+  uint32_t k4 = (a >> 13) & 0x7FFFCu;
+  if (CLAMP_HI) k4 = k4 > t.hi4 ? t.hi4 : k4;
+  const uint32_t e = fetch(k4);
+  return e + ((a << 17) > e ? 1u : 0u);
 }
 
 // Gathers the low bytes of four words into one word (word 0 in byte 0).
