@@ -91,6 +91,16 @@ int dt8_codebook(int is_signed, float *out_host);
  */
 int dt8_selfcheck_encode_host(int is_signed, const float *v_host, int64_t n, uint8_t *out_host);
 
+/*
+ * Diagnostic, device: out_i = s_i / N_i computed by the routine the kernels use for Eq. quant1's
+ * normalisation (a correctly rounded reciprocal of N and a residual correction; the IEEE division
+ * when N is 0 or outside 2^-76 .. 2^100).  The method needs the correctly rounded quotient for
+ * |s_i| <= N_i; this entry point lets a test compare the routine with the true quotient on
+ * operands of its choice.  No step, quantize or dequantize call uses it.
+ *   s, N   device, const float[n];   out  device, float[n]
+ */
+int dt8_selfcheck_divide(const float *s, const float *N, int64_t n, float *out, void *stream);
+
 /* Optional: upload the constant tables to the current device now (otherwise the first call does
  * it).  Blocking; call outside stream capture. */
 int dt8_init(void);

@@ -16,9 +16,10 @@ import torch
 
 __all__ = [
     "DT8Error", "lib_path", "load_library", "num_blocks",
-    "dt8_codebook", "dt8_selfcheck_encode_host", "dt8_init", "dt8_quantize_blockwise",
+    "dt8_codebook", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_init",
+    "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step", "dt8_adam_step", "dt8_sgd_step_multi",
-    "dt8_adam_step_multi", "new_state", "shard_blocks",
+    "dt8_adam_step_multi", "new_state", "shard_blocks", "PreparedTensorList",
     "DT8_F32", "DT8_BF16", "DT8_ADAM_BIAS_CORRECTION", "DT8_ADAM_DECOUPLED_WD", "DEFAULT_ADAM_FLAGS",
     "BLOCK_SIZES",
 ]
@@ -35,7 +36,7 @@ _lib = None
 
 EXPORTS = (
     "dt8_status_string", "dt8_last_cuda_error", "dt8_codebook", "dt8_selfcheck_encode_host",
-    "dt8_init", "dt8_quantize_blockwise", "dt8_dequantize_blockwise", "dt8_sgd_step",
+    "dt8_selfcheck_divide", "dt8_init", "dt8_quantize_blockwise", "dt8_dequantize_blockwise", "dt8_sgd_step",
     "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
 )
 
@@ -70,6 +71,7 @@ def load_library() -> ctypes.CDLL:
     lib.dt8_last_cuda_error.restype = i32
     lib.dt8_codebook.argtypes = [i32, vp]
     lib.dt8_selfcheck_encode_host.argtypes = [i32, vp, i64, vp]
+    lib.dt8_selfcheck_divide.argtypes = [vp, vp, i64, vp, vp]
     lib.dt8_init.argtypes = []
     lib.dt8_quantize_blockwise.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     lib.dt8_dequantize_blockwise.argtypes = [vp, vp, i64, i32, i32, vp, vp]
@@ -140,6 +142,19 @@ def dt8_selfcheck_encode_host(is_signed: bool, v: np.ndarray) -> np.ndarray:
 def dt8_init(device=None) -> None:
     with torch.cuda.device(device if device is not None else torch.cuda.current_device()):
         _check(load_library().dt8_init(), "dt8_init")
+
+
+def dt8_selfcheck_divide(s: torch.Tensor, N: torch.Tensor, out: Optional[torch.Tensor] = None,
+                         stream=None) -> torch.Tensor:
+    """Diagnostic: the kernels' normalising division applied to operand pairs (s_i, N_i)."""
+    if out is None:
+        out = torch.empty_like(s)
+    with torch.cuda.device(s.device):
+        st = load_library().dt8_selfcheck_divide(
+            _dev_tensor(s, torch.float32, "s"), _dev_tensor(N, torch.float32, "N"), s.numel(),
+            _dev_tensor(out, torch.float32, "out"), _stream_ptr(stream, s.device))
+    _check(st, "dt8_selfcheck_divide")
+    return out
 
 
 def new_state(n: int, block_size: int, signed: bool, device) -> tuple:
@@ -259,6 +274,49 @@ def dt8_adam_step_multi(ps, gs, m_codes, m_absmax, r_codes, r_absmax, lr, beta1,
             ctypes.cast(narr, ctypes.c_void_p), lr, beta1, beta2, eps, weight_decay, step, block_size,
             flags, _stream_ptr(stream, dev))
     _check(st, "dt8_adam_step_multi")
+
+
+class PreparedTensorList:
+    """Pointer arrays of a tensor list, marshalled once and reused for every step.
+
+    The step functions above rebuild the host pointer arrays on each call, which costs more host
+    time than the launch itself for a few hundred tensors.  The tensors of an optimizer are updated
+    in place, so their addresses do not change between steps: marshal them once here and call
+    ``adam_step`` / ``sgd_step`` per step.  The object keeps the tensors alive.  Gradients must be
+    written into the same gradient tensors before each step."""
+
+    def __init__(self, ps, gs, m_codes, m_absmax, r_codes=None, r_absmax=None):
+        if len(ps) == 0:
+            raise ValueError("empty tensor list")
+        self._keep = (list(ps), list(gs), list(m_codes), list(m_absmax),
+                      list(r_codes or []), list(r_absmax or []))
+        self.device, self.g_dtype, self._g, self._n = _multi_common(ps, gs)
+        self.num = len(ps)
+        self._p = _PtrList(ps, torch.float32, "p")
+        self._mc = _PtrList(m_codes, torch.uint8, "m_codes")
+        self._ma = _PtrList(m_absmax, torch.float32, "m_absmax")
+        self._rc = _PtrList(r_codes, torch.uint8, "r_codes") if r_codes is not None else None
+        self._ra = _PtrList(r_absmax, torch.float32, "r_absmax") if r_absmax is not None else None
+
+    def sgd_step(self, lr, momentum, weight_decay, step, block_size=2048, stream=None) -> None:
+        with torch.cuda.device(self.device):
+            st = load_library().dt8_sgd_step_multi(
+                self.num, self._p.ptr, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
+                self._mc.ptr, self._ma.ptr, ctypes.cast(self._n, ctypes.c_void_p), lr, momentum,
+                weight_decay, step, block_size, _stream_ptr(stream, self.device))
+        _check(st, "dt8_sgd_step_multi")
+
+    def adam_step(self, lr, beta1, beta2, eps, weight_decay, step, block_size=2048,
+                  flags=DEFAULT_ADAM_FLAGS, stream=None) -> None:
+        if self._rc is None or self._ra is None:
+            raise ValueError("this list was prepared without second-moment states")
+        with torch.cuda.device(self.device):
+            st = load_library().dt8_adam_step_multi(
+                self.num, self._p.ptr, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
+                self._mc.ptr, self._ma.ptr, self._rc.ptr, self._ra.ptr,
+                ctypes.cast(self._n, ctypes.c_void_p), lr, beta1, beta2, eps, weight_decay, step,
+                block_size, flags, _stream_ptr(stream, self.device))
+        _check(st, "dt8_adam_step_multi")
 
 
 def shard_blocks(num_blocks_total: int, rank: int, world_size: int) -> range:

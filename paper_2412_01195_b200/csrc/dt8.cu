@@ -347,6 +347,22 @@ int dt8_init(void) {
   return ensure_device(&di, &em);
 }
 
+int dt8_selfcheck_divide(const float* s, const float* N, int64_t n, float* out, void* stream) {
+  if (n < 0) return DT8_ERR_INVALID_ARG;
+  if (n == 0) return DT8_OK;
+  if (!s || !N || !out) return DT8_ERR_INVALID_ARG;
+  if (!aligned(s, 4) || !aligned(N, 4) || !aligned(out, 4)) return DT8_ERR_ALIGNMENT;
+  DeviceInfo di;
+  EncMeta em;
+  int rc = ensure_device(&di, &em);
+  if (rc != DT8_OK) return rc;
+  const int64_t ctas = (n + 255) / 256;
+  const int grid = static_cast<int>(ctas < 8 * di.sm_count ? ctas : 8 * di.sm_count);
+  divide_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(s, N, out, n);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
 int dt8_quantize_blockwise(const float* x, int64_t n, int block_size, int is_signed, uint8_t* codes,
                            float* absmax, void* stream) {
   if (n < 0) return DT8_ERR_INVALID_ARG;

@@ -97,6 +97,44 @@ def test_quantize_follows_true_division(signed):
     quant_roundtrip_check(torch.from_numpy(x.ravel()), B, signed)
 
 
+def test_normalising_division_is_correctly_rounded():
+    """Eq. quant1 divides: the kernels' reciprocal-and-correct routine must give the correctly
+    rounded quotient for every |s| <= N.  The true quotient is formed in binary64 and rounded once
+    (a quotient of two binary32 numbers never sits on a binary32 rounding boundary, so the double
+    rounding is exact).  Scaling s or N by a power of two only shifts exponents, so the operand
+    space is (mantissa of N) x (mantissa of s, two binades): all 2^23 mantissas of s are swept for
+    N with all-ones, all-zeros, sparse and random mantissas."""
+    rng = np.random.default_rng(5)
+    man_n = np.concatenate([
+        np.array([0, 1, 2, 3, 0x7FFFFF, 0x7FFFFE, 0x7FFFFD, 0x400000, 0x400001, 0x3FFFFF, 0x555555,
+                  0x2AAAAA, 0x7FF000, 0x000FFF, 0x600000, 0x200000], np.uint32),
+        rng.integers(0, 1 << 23, 24).astype(np.uint32)])
+    man_s = np.arange(1 << 23, dtype=np.uint32)
+    for mn in man_n:
+        N = np.array([0x3F800000 | int(mn)], np.uint32).view(F)[0]
+        for expo in (0x3F800000, 0x3F000000):                 # s in [1, 2) and [0.5, 1)
+            s = (man_s | np.uint32(expo)).view(F)
+            s = s[s <= N]
+            if s.size == 0:
+                continue
+            got = dt8.dt8_selfcheck_divide(torch.from_numpy(s).to(DEV),
+                                           torch.full((s.size,), float(N), device=DEV)).cpu().numpy()
+            ref = (s.astype(np.float64) / np.float64(N)).astype(F)
+            bad = np.nonzero(got != ref)[0]
+            assert bad.size == 0, (float(N).hex(), [float(x).hex() for x in s[bad[:4]]], got[bad[:4]], ref[bad[:4]])
+    # random operands over the whole exponent range, the IEEE branch (tiny and huge N) included
+    M = 1 << 22
+    Nr = (rng.uniform(1, 2, M) * 2.0 ** rng.integers(-120, 120, M)).astype(F)
+    sr = np.minimum((Nr.astype(np.float64) * rng.uniform(-1, 1, M)).astype(F), Nr)
+    got = dt8.dt8_selfcheck_divide(torch.from_numpy(sr).to(DEV), torch.from_numpy(Nr).to(DEV)).cpu().numpy()
+    with np.errstate(under="ignore"):
+        ref = (sr.astype(np.float64) / Nr.astype(np.float64)).astype(F)
+    assert np.array_equal(got, ref)
+    # all-zero block: 0 / 0 is taken as 0
+    z = torch.zeros(8, device=DEV)
+    assert torch.count_nonzero(dt8.dt8_selfcheck_divide(z, z)).item() == 0
+
+
 @pytest.mark.parametrize("signed", [True, False])
 def test_encoder_over_a_strided_sweep_of_all_floats(signed):
     """Blocks whose maximum is exactly 1, so the normalised value is the input itself: every 13th
