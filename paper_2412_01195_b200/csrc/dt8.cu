@@ -403,25 +403,16 @@ int dt8_dequantize_blockwise(const uint8_t* codes, const float* absmax, int64_t 
   if (rc != DT8_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t quads = (n + 3) / 4;
-  const int64_t per_cta = static_cast<int64_t>(kCtaThreads) * kDeqUnroll;
+  const int64_t per_cta = static_cast<int64_t>(kDeqThreads) * kDeqUnroll;
   const int64_t ctas = (quads + per_cta - 1) / per_cta;
-  const int grid = static_cast<int>(ctas < di.sm_count ? ctas : di.sm_count);
+  const int64_t resident = static_cast<int64_t>(kDeqCtasPerSm) * di.sm_count;
+  const int grid = static_cast<int>(ctas < resident ? ctas : resident);
   const int shift = log2_int(block_size);
-  cudaError_t e;
-  if (is_signed) {
-    const size_t smem = smem_bytes(em, true, false, true, false);
-    static std::atomic<uint64_t> smem_ok{0};
-    e = allow_smem(smem_ok, dequantize_kernel<true>, di.device, smem);
-    if (e != cudaSuccess) return cuda_fail(e);
-    dequantize_kernel<true><<<grid, kCtaThreads, smem, s>>>(codes, absmax, out, n, shift, em);
-  } else {
-    const size_t smem = smem_bytes(em, false, true, true, false);
-    static std::atomic<uint64_t> smem_ok{0};
-    e = allow_smem(smem_ok, dequantize_kernel<false>, di.device, smem);
-    if (e != cudaSuccess) return cuda_fail(e);
-    dequantize_kernel<false><<<grid, kCtaThreads, smem, s>>>(codes, absmax, out, n, shift, em);
-  }
-  e = cudaGetLastError();
+  if (is_signed)
+    dequantize_kernel<true><<<grid, kDeqThreads, kDeqSmemBytes, s>>>(codes, absmax, out, n, shift);
+  else
+    dequantize_kernel<false><<<grid, kDeqThreads, kDeqSmemBytes, s>>>(codes, absmax, out, n, shift);
+  const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
 
