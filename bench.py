@@ -32,6 +32,10 @@ UNIT = "GB/s"
 WORKLOAD = "adam8bit_flat_2^28_fp32grad_block2048_wd0.01_prewarm10"
 DATASHEET_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
+# DRAM bytes (read + write) of one launch of the fused Adam kernel on 2^26 elements, from the ncu
+# capture summarised in profiles/; traffic is proportional to the element count (every byte is
+# touched once), so it is scaled to the launch that is timed.  Set to None when the kernel changes.
+NCU_TRAFFIC_BYTES_2P26 = 671593728 + 351755520
 
 
 def algorithmic_bytes(n: int, block: int) -> int:
@@ -193,22 +197,30 @@ def run_dt8(args):
     torch.cuda.synchronize()
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_head = torch.cuda.Event(enable_timing=True)
+    head_steps = min(50, args.steps)       # the GPU lowers its SM clock after ~0.1 s under load
     e0.record()
-    for _ in range(args.steps):
+    for i in range(args.steps):
         step += 1
         dt8.dt8_adam_step(w, g, mc, ma, rc, ra, *hp, step, B)
+        if i + 1 == head_steps:
+            e_head.record()
     e1.record()
     torch.cuda.synchronize()
     barrier()
     clocks = sampler.stop()
     ms_total = max_over_ranks(e0.elapsed_time(e1), dev)
     ms_step = ms_total / args.steps
+    ms_head = max_over_ranks(e0.elapsed_time(e_head), dev) / head_steps
     launches = args.steps
 
     bytes_step = algorithmic_bytes(n, B)
     gbs_per_gpu = bytes_step / (ms_step * 1e-3) / 1e9
     value = gbs_per_gpu * world
     peak, peak_src = measured_peak()
+    traffic = args.traffic_bytes
+    if traffic is None and NCU_TRAFFIC_BYTES_2P26 is not None:
+        traffic = round(NCU_TRAFFIC_BYTES_2P26 * n / float(1 << 26))
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ------------
     e2e = run_e2e(dt8, torch, dev, n, B, hp, step, w, g, mc, ma, rc, ra, args, world)
@@ -228,10 +240,12 @@ def run_dt8(args):
         "e2e": e2e,
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": round(gbs_per_gpu, 2), "peak": peak, "unit": "GB/s",
-                     "frac": round(gbs_per_gpu / peak, 4), "traffic": args.traffic_bytes,
+                     "frac": round(gbs_per_gpu / peak, 4), "traffic": traffic,
                      "kernel": "dt8::block_kernel<AdamOp<2048,16,512,f32 grads,AdamW>,SingleArgs>",
                      "algorithmic_bytes_per_launch": bytes_step, "peak_source": peak_src,
-                     "per_launch_ms": round(ms_step, 5)},
+                     "per_launch_ms": round(ms_step, 5),
+                     "first_steps": {"steps": head_steps, "per_launch_ms": round(ms_head, 5),
+                                     "frac": round(bytes_step / (ms_head * 1e-3) / 1e9 / peak, 4)}},
     }
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:

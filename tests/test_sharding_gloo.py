@@ -1,0 +1,102 @@
+"""The multi-GPU path on CPU: world size 2 over gloo.
+
+The step shards on quantization-block boundaries with no exchange between ranks (Section IV-B:
+every block is quantized on its own).  These tests run the host-side logic of that path as two
+gloo ranks: the block partition, a sharded step that must equal the unsharded one bit for bit
+(each rank steps its own block range with the CPU checker), and the timing reduction the benchmark
+uses (barrier + maximum over ranks)."""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORLD = 2
+B = 256
+N = 37 * B + 91            # 38 blocks, the last one short
+HP = (1e-3, 0.9, 0.999, 1e-8, 0.01)
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _inputs():
+    from paper_2412_01195_b200 import synth
+    w, g = synth.flat_adam_inputs(N, 11)
+    return w.numpy().copy(), g.numpy().copy()
+
+
+def _worker(rank: int, port: int, out_dir: str):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      WORLD_SIZE=str(WORLD), LOCAL_RANK=str(rank))
+    dist.init_process_group("gloo", rank=rank, world_size=WORLD)
+    try:
+        import bench
+        import oracle
+        import paper_2412_01195_b200 as dt8
+
+        nb = dt8.num_blocks(N, B)
+        mine = dt8.shard_blocks(nb, rank, WORLD)
+        # 1. the partition: every block owned exactly once, ranges contiguous and ordered
+        owned = [None] * WORLD
+        dist.all_gather_object(owned, (mine.start, mine.stop))
+        assert owned[0][0] == 0 and owned[-1][1] == nb
+        assert all(owned[i][1] == owned[i + 1][0] for i in range(WORLD - 1))
+
+        # 2. a sharded step equals the unsharded step: each rank steps only its block range
+        w, g = _inputs()
+        lo, hi = mine.start * B, min(N, mine.stop * B)
+        ws, gs = w[lo:hi].copy(), g[lo:hi].copy()
+        n_loc = hi - lo
+        nb_loc = oracle.num_blocks(n_loc, B)
+        mc, ma = np.full(n_loc, 127, np.uint8), np.zeros(nb_loc, np.float32)
+        rc, ra = np.zeros(n_loc, np.uint8), np.zeros(nb_loc, np.float32)
+        for t in (1, 2, 3):
+            oracle.adam_step(ws, gs, mc, ma, rc, ra, *HP, t, B)
+        pieces = [None] * WORLD
+        dist.all_gather_object(pieces, (ws, mc, ma, rc, ra))
+        if rank == 0:
+            wf, gf = _inputs()
+            mcf, maf = np.full(N, 127, np.uint8), np.zeros(nb, np.float32)
+            rcf, raf = np.zeros(N, np.uint8), np.zeros(nb, np.float32)
+            for t in (1, 2, 3):
+                oracle.adam_step(wf, gf, mcf, maf, rcf, raf, *HP, t, B)
+            for k, full in enumerate((wf, mcf, maf, rcf, raf)):
+                joined = np.concatenate([p[k] for p in pieces])
+                assert np.array_equal(joined, full), f"sharded result {k} differs"
+
+        # 3. the benchmark's timing reduction: barrier, then the maximum over ranks
+        bench.barrier()
+        slowest = bench.max_over_ranks(10.0 * (rank + 1), torch.device("cpu"))
+        assert slowest == 10.0 * WORLD
+        with open(os.path.join(out_dir, f"ok{rank}"), "w") as fh:
+            fh.write("ok")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_shard_blocks_and_agree_with_the_unsharded_step(tmp_path):
+    mp.spawn(_worker, args=(_free_port(), str(tmp_path)), nprocs=WORLD, join=True)
+    assert all(os.path.exists(tmp_path / f"ok{r}") for r in range(WORLD))
+
+
+def test_reference_arm_runs_on_rank_zero_only(monkeypatch, capsys):
+    import bench
+    monkeypatch.setenv("RANK", "1")
+    monkeypatch.setenv("WORLD_SIZE", "2")
+
+    class Args:
+        steps, warmup = 1, 1
+    assert bench.run_reference(Args()) is None
+    assert capsys.readouterr().out == ""
