@@ -321,6 +321,84 @@ def test_multi_equals_single_and_skips_empty_tensors():
             assert torch.equal(u, v)
 
 
+def test_prepared_tensor_list_equals_the_per_call_form():
+    """Pointer arrays marshalled once give the same steps as arrays rebuilt on every call."""
+    B = 2048
+    sizes = [33, B, 5 * B + 77, 256, 9 * B]
+    hp = (1e-3, 0.9, 0.999, 1e-8, 0.05)
+    ws = [synth.normal(n, 0.02, 300 + i).to(DEV) for i, n in enumerate(sizes)]
+    gs = [synth.normal(n, 1e-3, 350 + i, dtype=torch.bfloat16).to(DEV) for i, n in enumerate(sizes)]
+    mk = lambda: [(w.clone(), *dt8.new_state(n, B, True, DEV), *dt8.new_state(n, B, False, DEV))
+                  for w, n in zip(ws, sizes)]
+    a, b = mk(), mk()
+    col = lambda rows, k: [r[k] for r in rows]
+    prepared = dt8.PreparedTensorList(col(a, 0), gs, col(a, 1), col(a, 2), col(a, 3), col(a, 4))
+    for t in (1, 2, 3, 4):
+        for g in gs:                                   # fresh gradients written in place
+            g.copy_(synth.normal(g.numel(), 1e-3, 400 + t, dtype=torch.bfloat16))
+        prepared.adam_step(*hp, t, B)
+        dt8.dt8_adam_step_multi(col(b, 0), gs, col(b, 1), col(b, 2), col(b, 3), col(b, 4), *hp, t, B)
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        for u, v in zip(x, y):
+            assert torch.equal(u, v)
+    sa, sb = mk(), mk()
+    gf = [g.float() for g in gs]
+    prepared = dt8.PreparedTensorList(col(sa, 0), gf, col(sa, 1), col(sa, 2))
+    for t in (1, 2):
+        prepared.sgd_step(0.1, 0.9, 1e-4, t, B)
+        dt8.dt8_sgd_step_multi(col(sb, 0), gf, col(sb, 1), col(sb, 2), 0.1, 0.9, 1e-4, t, B)
+    torch.cuda.synchronize()
+    for x, y in zip(sa, sb):
+        assert torch.equal(x[0], y[0]) and torch.equal(x[1], y[1]) and torch.equal(x[2], y[2])
+
+
+def test_non_finite_gradients_stay_inside_their_block():
+    """NaN / Inf are outside the contract, but they must not index outside the tables: a block
+    that holds one gets a non-finite maximum and takes the clamped path of the encoder.  Blocks
+    without one are unaffected (blocks are independent) and still match the CPU checker."""
+    B, nblk = 2048, 24
+    n = nblk * B
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    w0 = synth.normal(n, 0.02, 71)
+    g1 = synth.normal(n, 1e-3, 72)
+    g2 = synth.normal(n, 1e-3, 73)
+    bad_blocks = {3: float("nan"), 7: float("inf"), 11: float("-inf"), 12: float("nan")}
+    for blk, val in bad_blocks.items():
+        g2[blk * B + 5 * blk] = val
+    g2[12 * B + 1] = float("inf")
+    st = AdamState(w0, B)
+    st.step(g1, 1, hp)
+    st.check()
+    # second step with the poisoned gradient, on the GPU and in the checker
+    g2_gpu = g2.to(DEV)
+    dt8.dt8_adam_step(st.w_gpu, g2_gpu, st.mc_gpu, st.ma_gpu, st.rc_gpu, st.ra_gpu, hp["lr"],
+                      hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], 2, B)
+    w_sgd = w0.to(DEV).clone()
+    mc, ma = dt8.new_state(n, B, True, DEV)
+    dt8.dt8_sgd_step(w_sgd, g2_gpu, mc, ma, 0.1, 0.9, 1e-4, 1, B)
+    codes, absmax = dt8.dt8_quantize_blockwise(g2_gpu, B, True)
+    codes_u, _ = dt8.dt8_quantize_blockwise(g2_gpu, B, False)
+    torch.cuda.synchronize()                          # all four kernels ran to completion
+    with np.errstate(all="ignore"):
+        oracle.adam_step(st.w, to_np(g2), st.mc, st.ma, st.rc, st.ra, hp["lr"], hp["beta1"],
+                         hp["beta2"], hp["eps"], hp["weight_decay"], 2, B)
+        q_ref, a_ref = oracle.quantize_blockwise(to_np(g2), B, True)
+    good = np.ones(n, bool)
+    for blk in bad_blocks:
+        good[blk * B:(blk + 1) * B] = False
+    good_blk = np.array([b not in bad_blocks for b in range(nblk)])
+    assert np.array_equal(to_np(st.mc_gpu)[good], st.mc[good])
+    assert np.array_equal(to_np(st.rc_gpu)[good], st.rc[good])
+    assert np.array_equal(to_np(st.ma_gpu)[good_blk], st.ma[good_blk])
+    assert np.array_equal(to_np(st.ra_gpu)[good_blk], st.ra[good_blk])
+    assert_params_close(to_np(st.w_gpu)[good], st.w[good])
+    assert np.array_equal(to_np(codes)[good], q_ref[good])
+    assert np.array_equal(to_np(absmax)[good_blk], a_ref[good_blk])
+    assert not np.isfinite(to_np(st.ma_gpu)[~good_blk]).any()
+    assert codes_u.numel() == n
+
+
 def test_more_tensors_than_one_launch_holds():
     """600 small tensors: the pointer list is cut into several launches."""
     B = 256
