@@ -147,9 +147,11 @@ int dt8_sgd_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *
  *     p <- p - lr * (m'/bc1) / (sqrt(r'/bc2) + eps),  bc_i = 1 - beta_i^step, or 1 without bias
  *          correction
  *     m' is re-quantized with the signed table, r' with the unsigned table.
- * The parameter update uses the 32-bit m', r' before they are quantized.  With decoupled decay the
- * parameter update is evaluated with fast reciprocal / square root (relative error ~1e-7 of the
- * update); with coupled decay, where p feeds the states, it is evaluated with IEEE operations.
+ * The parameter update uses the 32-bit m', r' before they are quantized.  With decoupled decay, or
+ * with weight_decay == 0, the parameter update is evaluated with a single-instruction reciprocal
+ * and square root (relative error ~2e-7 of the update term); with coupled decay, where p feeds the
+ * states, and whenever eps*sqrt(bc2) < 1e-12 (a flushed subnormal root would show), it is
+ * evaluated with IEEE operations and is bit-reproducible against a plain binary32 evaluation.
  */
 int dt8_adam_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
                   uint8_t *r_codes, float *r_absmax, int64_t n, float lr, float beta1, float beta2,

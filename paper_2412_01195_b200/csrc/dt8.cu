@@ -280,8 +280,10 @@ AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float w
 // (below 1.1e-19) is invisible next to the scaled eps only while that is well above it.
 constexpr float kMinEpsForFastUpdate = 1e-12f;
 
+// Coupled decay makes the parameters an input of the states, so they must then be computed with
+// IEEE operations; without decay the two forms coincide and the fast parameter path applies.
 int adam_mode(uint32_t flags, const AdamHyper& h) {
-  if (!(flags & DT8_ADAM_DECOUPLED_WD)) return kAdamL2;
+  if (!(flags & DT8_ADAM_DECOUPLED_WD) && h.wd != 0.0f) return kAdamL2;
   return h.eps_scaled >= kMinEpsForFastUpdate ? kAdamWFast : kAdamWIeee;
 }
 

@@ -214,6 +214,22 @@ def test_adam_variants(flags):
     st.check(exact_params=not (flags & dt8.DT8_ADAM_DECOUPLED_WD))
 
 
+def test_adam_literal_equation_without_decay_and_tiny_eps():
+    """Eq. adam exactly as printed (no bias correction, no decay) takes the fast parameter path
+    (1e-6); an eps too small for that path takes IEEE operations (bit-exact parameters)."""
+    n, B = 21 * 2048 + 77, 2048
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    st = AdamState(synth.normal(n, 0.02, 610), B)
+    for t in range(1, 11):
+        st.step(synth.fresh_grad(n, 44, t), t, hp, 0)
+    st.check()
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-20, weight_decay=0.01)
+    st = AdamState(synth.normal(n, 0.02, 611), B)
+    for t in range(1, 6):
+        st.step(synth.fresh_grad(n, 45, t), t, hp)
+    st.check(exact_params=True)
+
+
 def test_adam_heavy_tailed_and_sparse_gradients():
     """Student-t gradients, zero gradients, and a block that stays all-zero."""
     hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
