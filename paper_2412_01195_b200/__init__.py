@@ -16,7 +16,7 @@ import torch
 
 __all__ = [
     "DT8Error", "lib_path", "load_library", "num_blocks",
-    "dt8_codebook", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_init",
+    "dt8_codebook", "dt8_state_bytes", "optimizer_state_bytes", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_init",
     "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step", "dt8_adam_step", "dt8_sgd_step_multi",
     "dt8_adam_step_multi", "new_state", "shard_blocks", "PreparedTensorList",
@@ -35,7 +35,8 @@ _LIB_PATH = os.path.join(_HERE, "libdt8.so")
 _lib = None
 
 EXPORTS = (
-    "dt8_status_string", "dt8_last_cuda_error", "dt8_codebook", "dt8_selfcheck_encode_host",
+    "dt8_status_string", "dt8_last_cuda_error", "dt8_codebook", "dt8_state_bytes",
+    "dt8_selfcheck_encode_host",
     "dt8_selfcheck_divide", "dt8_init", "dt8_quantize_blockwise", "dt8_dequantize_blockwise", "dt8_sgd_step",
     "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
 )
@@ -70,6 +71,8 @@ def load_library() -> ctypes.CDLL:
     lib.dt8_status_string.argtypes = [i32]
     lib.dt8_last_cuda_error.restype = i32
     lib.dt8_codebook.argtypes = [i32, vp]
+    lib.dt8_state_bytes.argtypes = [i64, i32]
+    lib.dt8_state_bytes.restype = i64
     lib.dt8_selfcheck_encode_host.argtypes = [i32, vp, i64, vp]
     lib.dt8_selfcheck_divide.argtypes = [vp, vp, i64, vp, vp]
     lib.dt8_init.argtypes = []
@@ -125,6 +128,22 @@ def dt8_codebook(is_signed: bool) -> np.ndarray:
     out = np.empty(256, np.float32)
     _check(load_library().dt8_codebook(int(bool(is_signed)), out.ctypes.data), "dt8_codebook")
     return out
+
+
+def dt8_state_bytes(n: int, block_size: int = 2048) -> int:
+    """Bytes of one 8-bit state of n elements (codes + one fp32 maximum per block)."""
+    b = load_library().dt8_state_bytes(n, block_size)
+    if b < 0:
+        raise ValueError("dt8_state_bytes: n >= 0 and a supported block size are required")
+    return int(b)
+
+
+def optimizer_state_bytes(sizes: Sequence[int], states_per_weight: int, block_size: int = 2048):
+    """(32-bit bytes, 8-bit bytes) of the optimizer state of a tensor list: SGD with momentum
+    keeps one state per weight, Adam two; every tensor is chunked on its own."""
+    full = 4 * states_per_weight * sum(int(n) for n in sizes)
+    small = states_per_weight * sum(dt8_state_bytes(int(n), block_size) for n in sizes)
+    return full, small
 
 
 def dt8_selfcheck_encode_host(is_signed: bool, v: np.ndarray) -> np.ndarray:

@@ -10,8 +10,6 @@
 #include "dt8_kernels.cuh"
 
 namespace dt8 {
-
-
 namespace {
 
 thread_local int tl_last_cuda_error = 0;
@@ -298,7 +296,7 @@ const char* dt8_status_string(int status) {
   switch (status) {
     case DT8_OK: return "DT8_OK";
     case DT8_ERR_INVALID_ARG: return "DT8_ERR_INVALID_ARG: bad pointer, size, step, dtype or flag";
-    case DT8_ERR_UNSUPPORTED: return "DT8_ERR_UNSUPPORTED: block size must be 256, 512, 1024, 2048 or 4096";
+    case DT8_ERR_UNSUPPORTED: return "DT8_ERR_UNSUPPORTED: block size must be 256, 512, 1024, 2048 or 4096 (or the device cannot hold the shared-memory table layout)";
     case DT8_ERR_ALIGNMENT: return "DT8_ERR_ALIGNMENT: fp32 tensors need 16-byte, bf16 8-byte, codes and absmax 4-byte alignment";
     case DT8_ERR_CUDA: return "DT8_ERR_CUDA: a CUDA runtime call failed (see dt8_last_cuda_error)";
   }
@@ -311,6 +309,11 @@ int dt8_codebook(int is_signed, float* out_host) {
   if (!out_host) return DT8_ERR_INVALID_ARG;
   build_codebook(is_signed != 0, out_host);
   return DT8_OK;
+}
+
+int64_t dt8_state_bytes(int64_t n, int block_size) {
+  if (n < 0 || !block_size_ok(block_size)) return -1;
+  return n + 4 * ((n + block_size - 1) / block_size);
 }
 
 int dt8_selfcheck_encode_host(int is_signed, const float* v_host, int64_t n, uint8_t* out_host) {

@@ -48,6 +48,26 @@ def test_codebook_is_bit_identical_to_the_checker(signed):
     assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
 
 
+def test_state_bytes_and_the_papers_saving(paper_facts):
+    """1 byte per element + 4 bytes per block; the paper's "75 %" on its own kind of tensor list."""
+    from paper_2412_01195_b200 import synth
+    assert dt8.dt8_state_bytes(0) == 0
+    assert dt8.dt8_state_bytes(1) == 5 and dt8.dt8_state_bytes(2048) == 2052
+    assert dt8.dt8_state_bytes(2049) == 2049 + 8 and dt8.dt8_state_bytes(256, 256) == 260
+    with pytest.raises(ValueError):
+        dt8.dt8_state_bytes(10, 1000)
+    flat_full, flat_small = dt8.optimizer_state_bytes([1 << 28], 2)
+    assert flat_full == paper_facts["adam_state_bytes_fp32"] * (1 << 28)
+    assert abs(100 * (1 - flat_small / flat_full) - 74.95) < 0.01
+    sizes = [synth.numel(s) for _, s, _ in synth.resnet_speaker_manifest()]
+    for states in (1, 2):                                  # SGD momentum, Adam
+        full, small = dt8.optimizer_state_bytes(sizes, states)
+        assert full == 4 * states * sum(sizes)
+        saving = 100 * (1 - small / full)
+        # small batch-norm vectors pay a whole absmax each, so a real list saves a little less
+        assert paper_facts["memory_saving_percent"] - 0.2 < saving < paper_facts["memory_saving_percent"]
+
+
 def test_codebook_null(lib):
     assert lib.dt8_codebook(1, None) == dt8.DT8_ERR_INVALID_ARG
 
