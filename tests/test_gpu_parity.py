@@ -415,6 +415,30 @@ def test_non_finite_gradients_stay_inside_their_block():
     assert codes_u.numel() == n
 
 
+def test_sharded_adam_on_one_rank_equals_the_plain_step():
+    """The block-range-sharded optimizer with a single rank (no process group) is the plain step
+    on a zero-padded buffer."""
+    from paper_2412_01195_b200.sharded import ShardedAdam8bit
+    n, B = 13 * 2048 + 300, 2048
+    hp = (1e-3, 0.9, 0.999, 1e-8, 0.01)
+    opt = ShardedAdam8bit(n, B, device=DEV)
+    w0 = synth.normal(n, 0.02, 31).to(DEV)
+    opt.params[:n].copy_(w0)
+    w = torch.zeros(opt.padded, device=DEV)
+    w[:n].copy_(w0)
+    mc, ma = dt8.new_state(opt.padded, B, True, DEV)
+    rc, ra = dt8.new_state(opt.padded, B, False, DEV)
+    for t in (1, 2, 3):
+        g = torch.zeros(opt.padded, device=DEV)
+        g[:n].copy_(synth.fresh_grad(n, 32, t))
+        opt.grads.copy_(g)
+        opt.step(*hp)
+        dt8.dt8_adam_step(w, g, mc, ma, rc, ra, *hp, t, B)
+    torch.cuda.synchronize()
+    assert torch.equal(opt.params, w) and torch.equal(opt.m_codes, mc) and torch.equal(opt.r_codes, rc)
+    assert torch.equal(opt.m_absmax, ma) and torch.equal(opt.r_absmax, ra)
+
+
 def test_more_tensors_than_one_launch_holds():
     """600 small tensors: the pointer list is cut into several launches."""
     B = 256

@@ -86,6 +86,60 @@ def _worker(rank: int, port: int, out_dir: str):
         dist.destroy_process_group()
 
 
+def _oracle_step(w, g, mc, ma, rc, ra, lr, b1, b2, eps, wd, step, block, flags):
+    """Stands in for the CUDA step on CPU tensors (their numpy views share memory)."""
+    import oracle
+    oracle.adam_step(w.numpy(), g.numpy(), mc.numpy(), ma.numpy(), rc.numpy(), ra.numpy(), lr, b1,
+                     b2, eps, wd, step, block, flags)
+
+
+def _sharded_worker(rank: int, port: int, out_dir: str):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      WORLD_SIZE=str(WORLD), LOCAL_RANK=str(rank))
+    dist.init_process_group("gloo", rank=rank, world_size=WORLD)
+    try:
+        import oracle
+        from paper_2412_01195_b200 import synth
+        from paper_2412_01195_b200.sharded import ShardedAdam8bit, shard_layout
+
+        blocks, per_rank, padded = shard_layout(N, B, WORLD)
+        assert per_rank == blocks * B and padded == WORLD * per_rank >= N
+        opt = ShardedAdam8bit(N, B, device="cpu", step_fn=_oracle_step)
+        w0 = synth.normal(N, 0.02, 21)
+        opt.params[:N].copy_(w0)
+        # reference: the unsharded step on the gradient averaged over the ranks
+        w_ref = np.zeros(padded, np.float32)
+        w_ref[:N] = w0.numpy()
+        nb = oracle.num_blocks(padded, B)
+        mc, ma = np.full(padded, 127, np.uint8), np.zeros(nb, np.float32)
+        rc, ra = np.zeros(padded, np.uint8), np.zeros(nb, np.float32)
+        for t in (1, 2, 3):
+            local = [synth.normal(N, 1e-3, 100 * t + r) for r in range(WORLD)]
+            opt.grads.zero_()
+            opt.grads[:N].copy_(local[rank])
+            opt.step(*HP)
+            mean = np.zeros(padded, np.float32)
+            mean[:N] = ((local[0] + local[1]) / WORLD).numpy()
+            oracle.adam_step(w_ref, mean, mc, ma, rc, ra, *HP, t, B)
+        assert np.array_equal(opt.params.numpy(), w_ref), "gathered parameters differ"
+        lo = rank * per_rank
+        assert np.array_equal(opt.m_codes.numpy(), mc[lo:lo + per_rank])
+        assert np.array_equal(opt.r_absmax.numpy(), ra[lo // B:(lo + per_rank) // B])
+        assert opt.state_bytes() == 2 * (per_rank + 4 * blocks)
+        with open(os.path.join(out_dir, f"ok{rank}"), "w") as fh:
+            fh.write("ok")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_sharded_adam_reduce_scatter_step_all_gather(tmp_path):
+    """reduce-scatter(grads) -> step on the owned blocks -> all-gather(params), two gloo ranks,
+    with the CPU checker standing in for the CUDA step: equals the unsharded step on the mean
+    gradient bit for bit."""
+    mp.spawn(_sharded_worker, args=(_free_port(), str(tmp_path)), nprocs=WORLD, join=True)
+    assert all(os.path.exists(tmp_path / f"ok{r}") for r in range(WORLD))
+
+
 def test_two_ranks_shard_blocks_and_agree_with_the_unsharded_step(tmp_path):
     mp.spawn(_worker, args=(_free_port(), str(tmp_path)), nprocs=WORLD, join=True)
     assert all(os.path.exists(tmp_path / f"ok{r}") for r in range(WORLD))
