@@ -159,15 +159,19 @@ def run_dt8(args):
     import torch
     import torch.distributed as dist
     import paper_2412_01195_b200 as dt8
+    from paper_2412_01195_b200 import build as dt8_build
     from paper_2412_01195_b200 import synth
 
     rank, local_rank, world = dist_env()
+    if local_rank == 0:
+        dt8_build.build_library()          # no-op when libdt8.so is newer than its sources
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; the dt8 path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()                     # the other ranks wait for rank 0's build check
     c = dict(synth.ADAM_FLAT_LARGE)
     n, B = (args.n or c["n"]), c["block_size"]
     hp = (c["lr"], c["beta1"], c["beta2"], c["eps"], c["weight_decay"])
