@@ -269,8 +269,10 @@ AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float w
     h.bc2 = 1.0f;
   }
   const double root_bc2 = std::sqrt(static_cast<double>(h.bc2));
-  h.step_scale = static_cast<float>(static_cast<double>(lr) * root_bc2 / static_cast<double>(h.bc1));
+  const double ss = static_cast<double>(lr) * root_bc2 / static_cast<double>(h.bc1);
   h.eps_scaled = static_cast<float>(static_cast<double>(eps) * root_bc2);
+  h.inv_step = static_cast<float>(1.0 / ss);
+  h.eps_over_step = static_cast<float>(static_cast<double>(eps) * root_bc2 / ss);
   return h;
 }
 
@@ -282,7 +284,11 @@ constexpr float kMinEpsForFastUpdate = 1e-12f;
 // IEEE operations; without decay the two forms coincide and the fast parameter path applies.
 int adam_mode(uint32_t flags, const AdamHyper& h) {
   if (!(flags & DT8_ADAM_DECOUPLED_WD) && h.wd != 0.0f) return kAdamL2;
-  return h.eps_scaled >= kMinEpsForFastUpdate ? kAdamWFast : kAdamWIeee;
+  // the fast path also divides by the step size, so that must be a normal, moderate number
+  const bool fast = h.eps_scaled >= kMinEpsForFastUpdate && h.lr >= 1e-20f && h.lr <= 1e20f &&
+                    std::isfinite(h.inv_step) && std::isfinite(h.eps_over_step) &&
+                    h.eps_over_step >= 1e-30f;
+  return fast ? kAdamWFast : kAdamWIeee;
 }
 
 }  // namespace
