@@ -6,12 +6,14 @@ Cases: adam adam26 adambf adambf26 adaml2 sgd sgd26 sgdbf blocks quant dequant m
 Each case runs the public binding in a loop of 50 launches after 5 warm-ups between two CUDA
 events on the launching stream and prints milliseconds per launch, effective GB/s (algorithmic
 bytes of the method divided by the time) and the fraction of a reference bandwidth (``--peak``,
-GB/s; default: the copy bandwidth measured on a B200).  Tensors are larger than the L2 cache
+GB/s; default: the measured copy bandwidth recorded for this machine, else 6650).  Tensors are larger than the L2 cache
 except in the tensor-list cases, which say so.
 """
 from __future__ import annotations
 
 import argparse
+import json
+import os
 
 import torch
 
@@ -157,8 +159,17 @@ def multi_cases(report, dev):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("cases", nargs="*", default=ALL)
-    ap.add_argument("--peak", type=float, default=6536.0, help="reference bandwidth in GB/s")
+    ap.add_argument("--peak", type=float, default=None,
+                    help="reference bandwidth in GB/s (default: hbm_gbs of MEASURED_PEAKS.json at the "
+                         "repository root if present, else 6650)")
     args = ap.parse_args()
+    if args.peak is None:
+        here = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+        try:
+            with open(os.path.join(here, "MEASURED_PEAKS.json")) as fh:
+                args.peak = float(json.load(fh)["hbm_gbs"])
+        except Exception:
+            args.peak = 6650.0
     if not torch.cuda.is_available():
         raise RuntimeError("needs a CUDA device: the dt8 library has no CPU path")
     dev = torch.device("cuda", torch.cuda.current_device())
