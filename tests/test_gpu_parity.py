@@ -439,6 +439,31 @@ def test_sharded_adam_on_one_rank_equals_the_plain_step():
     assert torch.equal(opt.m_absmax, ma) and torch.equal(opt.r_absmax, ra)
 
 
+def test_streamed_host_resident_step_equals_the_device_resident_step():
+    """Tensors in pinned host memory, streamed through the GPU in chunks of whole blocks on three
+    streams: bit-identical to stepping the whole tensor on the device (blocks are independent)."""
+    from paper_2412_01195_b200.offload import StreamedAdam8bit
+    B = 512
+    n = 37 * B + 123                              # 8 chunks of 5 blocks, the last one short and ragged
+    hp = (1e-3, 0.9, 0.999, 1e-8, 0.01)
+    w0 = synth.normal(n, 0.02, 81)
+    ref = [w0.to(DEV), None, *dt8.new_state(n, B, True, DEV), *dt8.new_state(n, B, False, DEV)]
+    host = [w0.clone().pin_memory(), torch.empty(n).pin_memory()]
+    host += [t.cpu().pin_memory() for t in ref[2:]]
+    pipe = StreamedAdam8bit(B, chunk_elems=5 * B + 17, buffers=2, device=DEV)
+    assert pipe.chunk == 5 * B
+    for t in (1, 2, 3):
+        g = synth.fresh_grad(n, 82, t)
+        host[1].copy_(g)
+        pipe.step(*host, *hp, t)
+        dt8.dt8_adam_step(ref[0], g.to(DEV), *ref[2:], *hp, t, B)
+    torch.cuda.synchronize()
+    assert pipe.h2d_bytes == n * 10 + 8 * dt8.num_blocks(n, B)
+    assert pipe.d2h_bytes == n * 6 + 8 * dt8.num_blocks(n, B)
+    for h, d in zip([host[0]] + host[2:], [ref[0]] + ref[2:]):
+        assert torch.equal(h, d.cpu())
+
+
 def test_more_tensors_than_one_launch_holds():
     """600 small tensors: the pointer list is cut into several launches."""
     B = 256
