@@ -26,7 +26,8 @@
  *     block b covers elements [b*block_size, min(n, (b+1)*block_size)).  `codes` holds n bytes,
  *     `absmax` holds nb floats (Section IV-B, "Tensor chunking").  Blocks never span tensors.
  *   - block_size is one of 256, 512, 1024, 2048, 4096 (the paper uses 2048), else
- *     DT8_ERR_UNSUPPORTED.
+ *     DT8_ERR_UNSUPPORTED.  A tensor may have at most 2^31 - 2^16 blocks (4.4e12 elements at
+ *     block_size 2048), else DT8_ERR_UNSUPPORTED.
  *   - Alignment: fp32 tensors 16 bytes, bf16 tensors 8 bytes, code arrays 4 bytes, absmax arrays
  *     4 bytes, at each tensor's base; else DT8_ERR_ALIGNMENT.
  *   - n == 0 (or num_tensors == 0) is a successful no-op.  n < 0, a NULL tensor pointer with

@@ -99,6 +99,9 @@ cudaError_t allow_smem(std::atomic<uint64_t>& done, K kernel, int device, size_t
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
+// The kernels index quantization blocks with 32 bits (next block = block + grid stride).
+constexpr int64_t kMaxBlocksPerLaunch = 0x7FFF0000;
+
 bool block_size_ok(int B) { return B == 256 || B == 512 || B == 1024 || B == 2048 || B == 4096; }
 
 int log2_int(int v) {
@@ -245,6 +248,7 @@ int launch_quantize(const float* x, int64_t n, uint8_t* codes, float* absmax, co
   SingleArgs a;
   a.t = TensorDesc{nullptr, x, codes, absmax, nullptr, nullptr, n};
   a.nb = (n + B - 1) / B;
+  if (a.nb > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
   kernel<<<grid_for(a.nb, GROUPS, di.sm_count), THREADS, smem, stream>>>(a, NoHyper{0}, em);
   e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
@@ -438,6 +442,7 @@ int dt8_sgd_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float* 
   int rc = check_tensor(a.t, g_dtype, false);
   if (rc != DT8_OK || n == 0) return rc;
   a.nb = (n + block_size - 1) / block_size;
+  if (a.nb > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
   DeviceInfo di;
   EncMeta em;
   rc = ensure_device(&di, &em);
@@ -458,6 +463,7 @@ int dt8_adam_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float*
   int rc = check_tensor(a.t, g_dtype, true);
   if (rc != DT8_OK || n == 0) return rc;
   a.nb = (n + block_size - 1) / block_size;
+  if (a.nb > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
   DeviceInfo di;
   EncMeta em;
   rc = ensure_device(&di, &em);
@@ -503,7 +509,7 @@ int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtyp
     while (i < num_tensors && args.num < kMaxTensorsPerLaunch) {
       if (n[i] > 0) {
         const int64_t nb = (n[i] + block_size - 1) / block_size;
-        if (blocks + nb > 0x7FFFFFFF) {
+        if (blocks + nb > kMaxBlocksPerLaunch) {
           if (args.num == 0) return DT8_ERR_UNSUPPORTED;
           break;
         }
