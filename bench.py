@@ -35,7 +35,7 @@ FALLBACK_PEAK_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the fused Adam kernel on 2^26 elements, from the ncu
 # capture summarised in profiles/; traffic is proportional to the element count (every byte is
 # touched once), so it is scaled to the launch that is timed.  Set to None when the kernel changes.
-NCU_TRAFFIC_BYTES_2P26 = 671458304 + 350965248
+NCU_TRAFFIC_BYTES_2P26 = 671457536 + 351272448
 
 
 def algorithmic_bytes(n: int, block: int) -> int:
