@@ -140,8 +140,13 @@ template <int B, int VPT_WANTED, int THREADS_WANTED> struct GeometryOf {
   static constexpr int THREADS = (THREADS_WANTED % (B / VPT) == 0) ? THREADS_WANTED : (B / VPT);
   static_assert(VPT % 4 == 0 && THREADS <= kCtaThreads && THREADS % (B / VPT) == 0, "bad geometry");
 };
-template <int B> using AdamGeometry = GeometryOf<B, DT8_ADAM_VPT, DT8_ADAM_THREADS>;
-template <int B> using SgdGeometry = GeometryOf<B, DT8_SGD_VPT, DT8_SGD_THREADS>;
+// Small blocks are latency-bound rather than issue-bound (one warp owns a block): 768 threads
+// with 8 values each measured 1-5 % faster there than 512 x 16.
+template <int B> struct AdamGeometry : GeometryOf<B, DT8_ADAM_VPT, DT8_ADAM_THREADS> {};
+template <> struct AdamGeometry<256> : GeometryOf<256, 8, 768> {};
+template <> struct AdamGeometry<512> : GeometryOf<512, 8, 768> {};
+template <int B> struct SgdGeometry : GeometryOf<B, DT8_SGD_VPT, DT8_SGD_THREADS> {};
+template <> struct SgdGeometry<256> : GeometryOf<256, 8, 768> {};
 template <int B> using QuantGeometry = GeometryOf<B, DT8_QUANT_VPT, DT8_QUANT_THREADS>;
 
 int check_tensor(const TensorDesc& d, int g_dtype, bool adam) {
