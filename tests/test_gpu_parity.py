@@ -464,6 +464,90 @@ def test_streamed_host_resident_step_equals_the_device_resident_step():
         assert torch.equal(h, d.cpu())
 
 
+def _tiny_speaker_net():
+    torch.manual_seed(0)
+    return torch.nn.Sequential(
+        torch.nn.Conv2d(1, 32, 3, padding=1), torch.nn.BatchNorm2d(32), torch.nn.ReLU(),
+        torch.nn.Conv2d(32, 64, 3, padding=1), torch.nn.BatchNorm2d(64), torch.nn.ReLU(),
+        torch.nn.AdaptiveAvgPool2d(1), torch.nn.Flatten(), torch.nn.Linear(64, 10)).to(DEV)
+
+
+@pytest.mark.parametrize("kind", ["adamw", "sgd"])
+def test_torch_optimizer_front_end_steps_and_resumes(kind):
+    """AdamW8bit / SGD8bit on a small conv net: every step equals the pointer-list entry point
+    called by hand on copies, and a run resumed from state_dict() continues bit-identically."""
+    from paper_2412_01195_b200.optim import AdamW8bit, SGD8bit
+
+    def make(model):
+        if kind == "adamw":
+            return AdamW8bit(model.parameters(), lr=1e-3, weight_decay=0.05, block_size=256)
+        return SGD8bit(model.parameters(), lr=0.05, momentum=0.9, weight_decay=1e-4, block_size=256)
+
+    def batch(i):
+        g = torch.Generator(device="cpu").manual_seed(100 + i)
+        return torch.randn(8, 1, 16, 16, generator=g).to(DEV), torch.randint(0, 10, (8,), generator=g).to(DEV)
+
+    def train(model, opt, steps):
+        # seeded gradients written in place (a real backward pass is not bit-reproducible run to
+        # run, which would hide what is being compared here: the optimizer)
+        for i in steps:
+            for k, prm in enumerate(model.parameters()):
+                g = synth.normal(prm.numel(), 1e-2, 7000 + 100 * i + k).view_as(prm).to(DEV)
+                if prm.grad is None:
+                    prm.grad = g
+                else:
+                    prm.grad.copy_(g)
+            opt.step()
+
+    # reference: the same gradients stepped by hand through the multi-tensor entry point
+    model = _tiny_speaker_net()
+    opt = make(model)
+    ps = [p.detach().clone() for p in model.parameters()]
+    B = 256
+    sm = [dt8.new_state(p.numel(), B, True, DEV) for p in ps]
+    sr = [dt8.new_state(p.numel(), B, False, DEV) for p in ps]
+    for i in range(1, 4):
+        x, y = batch(i)
+        opt.zero_grad(set_to_none=False)
+        torch.nn.functional.cross_entropy(model(x), y).backward()
+        gs = [p.grad.detach().clone() for p in model.parameters()]
+        opt.step()
+        flat = lambda ts: [t.view(-1) for t in ts]
+        if kind == "adamw":
+            dt8.dt8_adam_step_multi(flat(ps), flat(gs), [s[0] for s in sm], [s[1] for s in sm],
+                                    [s[0] for s in sr], [s[1] for s in sr], 1e-3, 0.9, 0.999, 1e-8,
+                                    0.05, i, B)
+        else:
+            dt8.dt8_sgd_step_multi(flat(ps), flat(gs), [s[0] for s in sm], [s[1] for s in sm], 0.05,
+                                   0.9, 1e-4, i, B)
+    torch.cuda.synchronize()
+    for p, q in zip(model.parameters(), ps):
+        assert torch.equal(p.detach(), q)
+    expected = sum(dt8.dt8_state_bytes(p.numel(), B) for p in ps) * (2 if kind == "adamw" else 1)
+    assert opt.state_bytes() == expected
+
+    # resume: 3 steps, checkpoint, 2 more steps == 5 steps in one go
+    a = _tiny_speaker_net()
+    oa = make(a)
+    train(a, oa, range(1, 6))
+    b = _tiny_speaker_net()
+    ob = make(b)
+    train(b, ob, range(1, 4))
+    ckpt = {"model": {k: v.clone() for k, v in b.state_dict().items()},
+            "opt": {"state": {i: {k: (v.clone() if torch.is_tensor(v) else v) for k, v in st.items()}
+                              for i, st in ob.state_dict()["state"].items()},
+                    "param_groups": ob.state_dict()["param_groups"]}}
+    c = _tiny_speaker_net()
+    c.load_state_dict(ckpt["model"])
+    oc = make(c)
+    oc.load_state_dict(ckpt["opt"])
+    assert all(st["m_codes"].dtype == torch.uint8 for st in oc.state.values())
+    train(c, oc, range(4, 6))
+    torch.cuda.synchronize()
+    for p, q in zip(a.parameters(), c.parameters()):
+        assert torch.equal(p.detach(), q.detach())
+
+
 def test_more_tensors_than_one_launch_holds():
     """600 small tensors: the pointer list is cut into several launches."""
     B = 256
