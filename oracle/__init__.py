@@ -32,16 +32,29 @@ _lock = threading.Lock()
 _lib = None
 
 
+def _compile(src: str, out: str) -> None:
+    tmp = out + ".%d.tmp" % os.getpid()
+    cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+           "-shared", "-fPIC", "-o", tmp, src, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, out)
+
+
 def build(force: bool = False) -> str:
-    """Compile the C oracle with gcc (no contraction, no fast-math) and return the .so path."""
+    """Compile the C oracle with gcc (no contraction, no fast-math) and return the .so path.
+
+    The mutation tests set DT8_ORACLE_SOURCE to a deliberately broken copy of the C file to show
+    that the pins notice it; that copy is built into a file of its own and never replaces the
+    real library."""
     os.makedirs(_OUT_DIR, exist_ok=True)
+    variant = os.environ.get("DT8_ORACLE_SOURCE")
+    if variant:
+        out = os.path.join(_OUT_DIR, "variant_%d.so" % os.getpid())
+        _compile(variant, out)
+        return out
     stale = (not os.path.exists(_SO)) or os.path.getmtime(_SO) < os.path.getmtime(_SRC)
     if force or stale:
-        tmp = _SO + ".%d.tmp" % os.getpid()
-        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
-               "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
-        subprocess.run(cmd, check=True)
-        os.replace(tmp, _SO)
+        _compile(_SRC, _SO)
     return _SO
 
 
