@@ -12,7 +12,9 @@
  *
  * Conventions shared by every entry point
  *   - Return value: a dt8_status.  On any status other than DT8_OK nothing was launched and no
- *     caller buffer was written.
+ *     caller buffer was written, with one exception: a pointer-list call that needs several
+ *     launches (more than 256 tensors) can return DT8_ERR_CUDA from a later launch after the
+ *     earlier ones were queued.  Every argument check is made before the first launch.
  *   - "device" pointers are CUDA device pointers of the current device, owned by the caller and
  *     valid until the work queued on `stream` has run.  "host" pointers are ordinary host memory.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the default
@@ -27,14 +29,16 @@
  *     `absmax` holds nb floats (Section IV-B, "Tensor chunking").  Blocks never span tensors.
  *   - block_size is one of 256, 512, 1024, 2048, 4096 (the paper uses 2048), else
  *     DT8_ERR_UNSUPPORTED.  A tensor may have at most 2^31 - 2^16 blocks (4.4e12 elements at
- *     block_size 2048), else DT8_ERR_UNSUPPORTED.
+ *     block_size 2048), in the single-tensor and the pointer-list forms alike, else
+ *     DT8_ERR_UNSUPPORTED.
  *   - Alignment: fp32 tensors 16 bytes, bf16 tensors 8 bytes, code arrays 4 bytes, absmax arrays
  *     4 bytes, at each tensor's base; else DT8_ERR_ALIGNMENT.
  *   - n == 0 (or num_tensors == 0) is a successful no-op.  n < 0, a NULL tensor pointer with
- *     n > 0, step < 1, or an unknown dtype / flag gives DT8_ERR_INVALID_ARG.
+ *     n > 0, step < 1, or an unknown dtype / flag gives DT8_ERR_INVALID_ARG.  So do non-finite
+ *     hyper-parameters, beta1 or beta2 outside [0, 1), a negative eps and a negative momentum.
  *   - A state whose absmax entries are all 0 is the zero state (Eq. adam: r_0 = m_0 = 0); its code
  *     bytes are then ignored on input.
- *   - Codes are indices into the ASCENDING table ("the integer index i corresponding to q_i").
+ *   - Codes are indices into the ASCENDING table (Section IV-B, "Indexing").
  *     The signed table has two zero entries, 127 and 128; the quantizer emits 127.
  *   - Arithmetic: everything that decides a code -- dequantized state, new state, block maximum,
  *     normalised value -- is computed in IEEE binary32, one rounding per written operation, no
@@ -113,6 +117,18 @@ int dt8_selfcheck_encode_host(int is_signed, const float *v_host, int64_t n, uin
  *   s, N   device, const float[n];   out  device, float[n]
  */
 int dt8_selfcheck_divide(const float *s, const float *N, int64_t n, float *out, void *stream);
+
+/*
+ * Diagnostic, device: out_i = s_i / d computed by the routine the IEEE form of the Adam parameter
+ * update uses for Eq. adam's bias corrections m'/(1 - beta1^step), r'/(1 - beta2^step), whose
+ * divisor is one number per launch: the host supplies the correctly rounded reciprocal of d and
+ * the kernel corrects the product with two fused multiply-adds; for d outside 2^-20 .. 2^20 or
+ * |s_i| outside 2^-60 .. 2^60 (zero included) it is the IEEE division.  The result must equal the
+ * correctly rounded quotient; this entry point lets a test check that on divisors and dividends
+ * of its choice.  No step, quantize or dequantize call uses it.
+ *   s  device, const float[n];   d  the divisor;   out  device, float[n]
+ */
+int dt8_selfcheck_divide_const(const float *s, float d, int64_t n, float *out, void *stream);
 
 /* Optional: upload the constant tables to the current device now (otherwise the first call does
  * it).  Blocking; call outside stream capture. */

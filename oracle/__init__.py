@@ -40,22 +40,31 @@ def _compile(src: str, out: str) -> None:
     os.replace(tmp, out)
 
 
-def build(force: bool = False) -> str:
-    """Compile the C oracle with gcc (no contraction, no fast-math) and return the .so path.
+def build_source(src: str, name: str, variant_env: str, force: bool = False) -> str:
+    """Compile one C file of the checker with gcc (no contraction, no fast-math) and return the
+    .so path.
 
-    The mutation tests set DT8_ORACLE_SOURCE to a deliberately broken copy of the C file to show
-    that the pins notice it; that copy is built into a file of its own and never replaces the
-    real library."""
-    os.makedirs(_OUT_DIR, exist_ok=True)
-    variant = os.environ.get("DT8_ORACLE_SOURCE")
+    The mutation tests set `variant_env` to a deliberately broken copy of the C file to show that
+    the pins notice it; that copy is built next to itself (in the test's temporary directory) and
+    never replaces the real library."""
+    variant = os.environ.get(variant_env)
     if variant:
-        out = os.path.join(_OUT_DIR, "variant_%d.so" % os.getpid())
+        out = os.path.splitext(variant)[0] + ".%d.so" % os.getpid()
         _compile(variant, out)
         return out
-    stale = (not os.path.exists(_SO)) or os.path.getmtime(_SO) < os.path.getmtime(_SRC)
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    out = os.path.join(_OUT_DIR, name)
+    stale = (not os.path.exists(out)) or os.path.getmtime(out) < os.path.getmtime(src)
     if force or stale:
-        _compile(_SRC, _SO)
-    return _SO
+        _compile(src, out)
+    return out
+
+
+def build(force: bool = False) -> str:
+    """Build every C file of the checker; returns the path of the optimizer checker's library."""
+    from . import rev
+    rev.build(force)
+    return build_source(_SRC, "libdt8_oracle.so", "DT8_ORACLE_SOURCE", force)
 
 
 def _load():
@@ -79,6 +88,12 @@ def _load():
             lib.dt8o_adam_step.argtypes = [fp, vp, c.c_int, u8p, fp, u8p, fp, c.c_int64, c.c_float,
                                            c.c_float, c.c_float, c.c_float, c.c_float, c.c_int64,
                                            c.c_int, c.c_uint32]
+            lib.dt8o_sgd_step_ex.argtypes = [vp, c.c_int, vp, c.c_int, u8p, fp, c.c_int64, c.c_float,
+                                             c.c_float, c.c_float, c.c_int64, c.c_int]
+            lib.dt8o_adam_step_ex.argtypes = [vp, c.c_int, vp, c.c_int, u8p, fp, u8p, fp, c.c_int64,
+                                              c.c_float, c.c_float, c.c_float, c.c_float, c.c_float,
+                                              c.c_int64, c.c_int, c.c_uint32]
+            lib.dt8o_bf16_round_many.argtypes = [fp, c.c_int64, vp]
             _lib = lib
     return _lib
 
@@ -174,28 +189,49 @@ def adam_update_fp32(w, g, m, r, lr, beta1, beta2, eps, weight_decay, step,
                                   lr, beta1, beta2, eps, weight_decay, step, flags)
 
 
+def bf16_round(x) -> np.ndarray:
+    """binary32 -> bfloat16 bit patterns (uint16), round to nearest even, element by element."""
+    x = np.ascontiguousarray(x, np.float32).ravel()
+    out = np.empty(x.size, np.uint16)
+    _load().dt8o_bf16_round_many(_f32(x, "x"), x.size, out.ctypes.data_as(ctypes.c_void_p))
+    return out
+
+
+def _param(w):
+    """fp32 ndarray, or bf16 bit patterns as a uint16 ndarray (the variant without a 32-bit copy)."""
+    if not (isinstance(w, np.ndarray) and w.flags.c_contiguous):
+        raise TypeError("w: need a C-contiguous ndarray")
+    if w.dtype == np.float32:
+        return w.ctypes.data_as(ctypes.c_void_p), F32
+    if w.dtype == np.uint16:
+        return w.ctypes.data_as(ctypes.c_void_p), BF16
+    raise TypeError("w: float32, or uint16 holding bfloat16 bit patterns")
+
+
 def sgd_step(w, g, m_codes, m_absmax, lr, momentum, weight_decay, step, block_size):
-    """One 8-bit SGD step, in place on w, m_codes, m_absmax."""
+    """One 8-bit SGD step, in place on w (fp32, or bf16 bit patterns), m_codes, m_absmax."""
     gp, gd = _grad(g)
+    wp, wd_ = _param(w)
     assert g.size == w.size == m_codes.size and m_absmax.size == num_blocks(w.size, block_size)
-    rc = _load().dt8o_sgd_step(_f32(w, "w"), gp, gd, _u8(m_codes, "m_codes"),
-                               _f32(m_absmax, "m_absmax"), w.size, lr, momentum, weight_decay,
-                               step, block_size)
+    rc = _load().dt8o_sgd_step_ex(wp, wd_, gp, gd, _u8(m_codes, "m_codes"),
+                                  _f32(m_absmax, "m_absmax"), w.size, lr, momentum, weight_decay,
+                                  step, block_size)
     if rc:
         raise ValueError("oracle sgd_step: bad arguments")
 
 
 def adam_step(w, g, m_codes, m_absmax, r_codes, r_absmax, lr, beta1, beta2, eps, weight_decay,
               step, block_size, flags=DEFAULT_ADAM_FLAGS):
-    """One 8-bit Adam/AdamW step, in place on w and both quantized states."""
+    """One 8-bit Adam/AdamW step, in place on w (fp32, or bf16 bit patterns) and both states."""
     gp, gd = _grad(g)
+    wp, wd_ = _param(w)
     nb = num_blocks(w.size, block_size)
     assert g.size == w.size == m_codes.size == r_codes.size
     assert m_absmax.size == nb and r_absmax.size == nb
-    rc = _load().dt8o_adam_step(_f32(w, "w"), gp, gd, _u8(m_codes, "m_codes"),
-                                _f32(m_absmax, "m_absmax"), _u8(r_codes, "r_codes"),
-                                _f32(r_absmax, "r_absmax"), w.size, lr, beta1, beta2, eps,
-                                weight_decay, step, block_size, flags)
+    rc = _load().dt8o_adam_step_ex(wp, wd_, gp, gd, _u8(m_codes, "m_codes"),
+                                   _f32(m_absmax, "m_absmax"), _u8(r_codes, "r_codes"),
+                                   _f32(r_absmax, "r_absmax"), w.size, lr, beta1, beta2, eps,
+                                   weight_decay, step, block_size, flags)
     if rc:
         raise ValueError("oracle adam_step: bad arguments")
 

@@ -42,7 +42,7 @@
 static int g_threads = 1;
 
 /* Number of host threads used for the loop over quantization blocks (blocks are
- * independent: Section IV-B, "quantization applied independently to each block"). */
+ * independent: each is quantized on its own, Section IV-B "Tensor chunking"). */
 void dt8o_set_threads(int t) { g_threads = t < 1 ? 1 : t; }
 int dt8o_get_threads(void) {
 #ifdef _OPENMP
@@ -65,7 +65,8 @@ int dt8o_get_threads(void) {
  *
  * evaluated as one binary64 division of two exact integers and rounded once to
  * binary32.  The all-zero field is the value 0.  The stored code is the index into
- * the ASCENDING table ("store the integer index i corresponding to q_i").
+ * the ASCENDING table (Section IV-B, "Indexing": what is stored is the position i
+ * of the chosen value q_i).
  * Signed table: out[127-p] = -value(p), out[128+p] = +value(p) for magnitude pattern
  * p (p = 0 is the value 0, so out[127] = out[128] = 0: the sign bit gives two zeros).
  * Unsigned table: out[p] = value(p).
@@ -112,7 +113,7 @@ uint8_t dt8o_nearest_scan(const float *Q, float v) {
 }
 
 /* The same decision by bisection over the sorted table, the search the paper names
- * ("binary search within the real-number domain D").  Finds the last entry <= v,
+ * (Section IV-B, "Nearest value searching").  Finds the last entry <= v,
  * compares it with its upper neighbour, and returns the lowest index holding the
  * chosen value. */
 uint8_t dt8o_nearest_bsearch(const float *Q, float v) {
@@ -212,6 +213,34 @@ static float grad_at(const void *g, int g_dtype, int64_t i) {
   return g_dtype == 0 ? ((const float *)g)[i] : bf16_widen(((const uint16_t *)g)[i]);
 }
 
+/* binary32 -> bfloat16, round to nearest, ties to even: the value is cut after the 8th
+ * significand bit; the 16 dropped bits decide (more than half: up; exactly half: to the even
+ * neighbour).  A NaN keeps its top bits with the quiet bit set. */
+uint16_t dt8o_bf16_round(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return (uint16_t)((u >> 16) | 0x0040u);
+  uint32_t kept = u >> 16, dropped = u & 0xFFFFu;
+  if (dropped > 0x8000u || (dropped == 0x8000u && (kept & 1u))) kept += 1;
+  return (uint16_t)kept;
+}
+
+void dt8o_bf16_round_many(const float *x, int64_t n, uint16_t *out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = dt8o_bf16_round(x[i]);
+}
+
+/* Parameters are binary32 in the paper (Section II: 32-bit floating point).  The bfloat16
+ * parameter variant (no 32-bit master copy) is a reading: the stored parameter is widened
+ * exactly, the update of Eq. sgd / Eq. adam runs in binary32 as written, and the result is
+ * rounded once, to nearest even, when it is stored. */
+static float param_at(const void *w, int p_dtype, int64_t i) {
+  return p_dtype == 0 ? ((const float *)w)[i] : bf16_widen(((const uint16_t *)w)[i]);
+}
+static void param_store(void *w, int p_dtype, int64_t i, float v) {
+  if (p_dtype == 0) ((float *)w)[i] = v;
+  else ((uint16_t *)w)[i] = dt8o_bf16_round(v);
+}
+
 /* ------------------------------------------------------------------------------
  * Eq. sgd on exact binary32 state (no quantizer):
  *     g' = g + wd*w      (weight decay as in the training recipe of Section V; skipped
@@ -280,8 +309,8 @@ void dt8o_adam_update_fp32(float *w, const float *g, float *m, float *r, int64_t
  * 8-bit SGD step (Section I / IV-B: states 8-bit -> 32-bit, weight update in 32-bit
  * with the 32-bit states, states quantized back with a fresh absmax).
  * ------------------------------------------------------------------------------ */
-int dt8o_sgd_step(float *w, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
-                  int64_t n, float lr, float beta, float wd, int64_t step, int B) {
+int dt8o_sgd_step_ex(void *w, int p_dtype, const void *g, int g_dtype, uint8_t *m_codes,
+                     float *m_absmax, int64_t n, float lr, float beta, float wd, int64_t step, int B) {
   (void)step;
   if (n < 0 || !block_size_ok(B)) return 1;
   float Qs[256];
@@ -295,21 +324,31 @@ int dt8o_sgd_step(float *w, const void *g, int g_dtype, uint8_t *m_codes, float 
     int cnt = (int)((n - s < B) ? (n - s) : B);
     float *m = (float *)malloc(sizeof(float) * (size_t)cnt);
     float *gb = (float *)malloc(sizeof(float) * (size_t)cnt);
+    float *wb = (float *)malloc(sizeof(float) * (size_t)cnt);
     for (int i = 0; i < cnt; ++i) gb[i] = grad_at(g, g_dtype, s + i);
+    for (int i = 0; i < cnt; ++i) wb[i] = param_at(w, p_dtype, s + i);
     dequantize_block(Qs, m_codes + s, m_absmax[b], cnt, m);
-    dt8o_sgd_update_fp32(w + s, gb, m, cnt, lr, beta, wd);
+    dt8o_sgd_update_fp32(wb, gb, m, cnt, lr, beta, wd);
     quantize_block(Qs, m, cnt, 0, m_codes + s, m_absmax + b);
+    for (int i = 0; i < cnt; ++i) param_store(w, p_dtype, s + i, wb[i]);
     free(m);
     free(gb);
+    free(wb);
   }
   return 0;
 }
 
+int dt8o_sgd_step(float *w, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
+                  int64_t n, float lr, float beta, float wd, int64_t step, int B) {
+  return dt8o_sgd_step_ex(w, 0, g, g_dtype, m_codes, m_absmax, n, lr, beta, wd, step, B);
+}
+
 /* 8-bit Adam / AdamW step: first moment on the signed table, second moment on the
  * unsigned table. */
-int dt8o_adam_step(float *w, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
-                   uint8_t *r_codes, float *r_absmax, int64_t n, float lr, float beta1,
-                   float beta2, float eps, float wd, int64_t step, int B, uint32_t flags) {
+int dt8o_adam_step_ex(void *w, int p_dtype, const void *g, int g_dtype, uint8_t *m_codes,
+                      float *m_absmax, uint8_t *r_codes, float *r_absmax, int64_t n, float lr,
+                      float beta1, float beta2, float eps, float wd, int64_t step, int B,
+                      uint32_t flags) {
   if (n < 0 || !block_size_ok(B) || step < 1) return 1;
   float Qs[256], Qu[256];
   dt8o_codebook(1, Qs);
@@ -324,15 +363,26 @@ int dt8o_adam_step(float *w, const void *g, int g_dtype, uint8_t *m_codes, float
     float *m = (float *)malloc(sizeof(float) * (size_t)cnt);
     float *r = (float *)malloc(sizeof(float) * (size_t)cnt);
     float *gb = (float *)malloc(sizeof(float) * (size_t)cnt);
+    float *wb = (float *)malloc(sizeof(float) * (size_t)cnt);
     for (int i = 0; i < cnt; ++i) gb[i] = grad_at(g, g_dtype, s + i);
+    for (int i = 0; i < cnt; ++i) wb[i] = param_at(w, p_dtype, s + i);
     dequantize_block(Qs, m_codes + s, m_absmax[b], cnt, m);
     dequantize_block(Qu, r_codes + s, r_absmax[b], cnt, r);
-    dt8o_adam_update_fp32(w + s, gb, m, r, cnt, lr, beta1, beta2, eps, wd, step, flags);
+    dt8o_adam_update_fp32(wb, gb, m, r, cnt, lr, beta1, beta2, eps, wd, step, flags);
     quantize_block(Qs, m, cnt, 0, m_codes + s, m_absmax + b);
     quantize_block(Qu, r, cnt, 0, r_codes + s, r_absmax + b);
+    for (int i = 0; i < cnt; ++i) param_store(w, p_dtype, s + i, wb[i]);
     free(m);
     free(r);
     free(gb);
+    free(wb);
   }
   return 0;
+}
+
+int dt8o_adam_step(float *w, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
+                   uint8_t *r_codes, float *r_absmax, int64_t n, float lr, float beta1,
+                   float beta2, float eps, float wd, int64_t step, int B, uint32_t flags) {
+  return dt8o_adam_step_ex(w, 0, g, g_dtype, m_codes, m_absmax, r_codes, r_absmax, n, lr, beta1,
+                           beta2, eps, wd, step, B, flags);
 }

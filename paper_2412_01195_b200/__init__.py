@@ -16,7 +16,7 @@ import torch
 
 __all__ = [
     "DT8Error", "lib_path", "load_library", "num_blocks",
-    "dt8_codebook", "dt8_state_bytes", "optimizer_state_bytes", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_init",
+    "dt8_codebook", "dt8_state_bytes", "optimizer_state_bytes", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_init",
     "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step", "dt8_adam_step", "dt8_sgd_step_multi",
     "dt8_adam_step_multi", "new_state", "shard_blocks", "PreparedTensorList",
@@ -37,7 +37,8 @@ _lib = None
 EXPORTS = (
     "dt8_status_string", "dt8_last_cuda_error", "dt8_codebook", "dt8_state_bytes",
     "dt8_selfcheck_encode_host",
-    "dt8_selfcheck_divide", "dt8_init", "dt8_quantize_blockwise", "dt8_dequantize_blockwise", "dt8_sgd_step",
+    "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_init", "dt8_quantize_blockwise",
+    "dt8_dequantize_blockwise", "dt8_sgd_step",
     "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
 )
 
@@ -75,6 +76,7 @@ def load_library() -> ctypes.CDLL:
     lib.dt8_state_bytes.restype = i64
     lib.dt8_selfcheck_encode_host.argtypes = [i32, vp, i64, vp]
     lib.dt8_selfcheck_divide.argtypes = [vp, vp, i64, vp, vp]
+    lib.dt8_selfcheck_divide_const.argtypes = [vp, f32, i64, vp, vp]
     lib.dt8_init.argtypes = []
     lib.dt8_quantize_blockwise.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     lib.dt8_dequantize_blockwise.argtypes = [vp, vp, i64, i32, i32, vp, vp]
@@ -108,6 +110,25 @@ def _dev_tensor(t: torch.Tensor, dtype, name: str) -> int:
     if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
         raise TypeError(f"{name}: need a contiguous CUDA tensor of dtype {dtype}")
     return t.data_ptr()
+
+
+def _check_layout(where: str, n: int, block_size: int, device, by_elements: dict, by_blocks: dict) -> None:
+    """The C ABI takes n and block_size on trust; the tensors' own sizes are known here.  A state
+    built for another block size, a gradient of another length or a tensor on another device would
+    make the kernel read or write outside an allocation, so each is refused before the call."""
+    if block_size not in BLOCK_SIZES:
+        raise ValueError(f"{where}: block_size must be one of {BLOCK_SIZES}")
+    nb = num_blocks(n, block_size)
+    for name, t in by_elements.items():
+        if t.numel() != n:
+            raise ValueError(f"{where}: {name} holds {t.numel()} elements, expected {n}")
+    for name, t in by_blocks.items():
+        if t.numel() != nb:
+            raise ValueError(f"{where}: {name} holds {t.numel()} block maxima, expected {nb} "
+                             f"(= ceil({n} / {block_size}))")
+    for name, t in {**by_elements, **by_blocks}.items():
+        if t.device != device:
+            raise ValueError(f"{where}: {name} is on {t.device}, expected {device}")
 
 
 def _grad_ptr(g: torch.Tensor):
@@ -176,6 +197,19 @@ def dt8_selfcheck_divide(s: torch.Tensor, N: torch.Tensor, out: Optional[torch.T
     return out
 
 
+def dt8_selfcheck_divide_const(s: torch.Tensor, d: float, out: Optional[torch.Tensor] = None,
+                               stream=None) -> torch.Tensor:
+    """Diagnostic: the constant-divisor division of the IEEE Adam update applied to (s_i, d)."""
+    if out is None:
+        out = torch.empty_like(s)
+    with torch.cuda.device(s.device):
+        st = load_library().dt8_selfcheck_divide_const(
+            _dev_tensor(s, torch.float32, "s"), float(d), s.numel(),
+            _dev_tensor(out, torch.float32, "out"), _stream_ptr(stream, s.device))
+    _check(st, "dt8_selfcheck_divide_const")
+    return out
+
+
 def new_state(n: int, block_size: int, signed: bool, device) -> tuple:
     """Zero state: canonical zero codes and absmax 0."""
     codes = torch.full((n,), 127 if signed else 0, dtype=torch.uint8, device=device)
@@ -187,10 +221,13 @@ def dt8_quantize_blockwise(x: torch.Tensor, block_size: int, is_signed: bool,
                            codes: Optional[torch.Tensor] = None, absmax: Optional[torch.Tensor] = None,
                            stream=None):
     n = x.numel()
+    if block_size not in BLOCK_SIZES:
+        raise ValueError(f"dt8_quantize_blockwise: block_size must be one of {BLOCK_SIZES}")
     if codes is None:
         codes = torch.empty(n, dtype=torch.uint8, device=x.device)
     if absmax is None:
         absmax = torch.empty(num_blocks(n, block_size), dtype=torch.float32, device=x.device)
+    _check_layout("dt8_quantize_blockwise", n, block_size, x.device, {"codes": codes}, {"absmax": absmax})
     with torch.cuda.device(x.device):
         st = load_library().dt8_quantize_blockwise(
             _dev_tensor(x, torch.float32, "x"), n, block_size, int(bool(is_signed)),
@@ -205,6 +242,7 @@ def dt8_dequantize_blockwise(codes: torch.Tensor, absmax: torch.Tensor, block_si
     n = codes.numel()
     if out is None:
         out = torch.empty(n, dtype=torch.float32, device=codes.device)
+    _check_layout("dt8_dequantize_blockwise", n, block_size, codes.device, {"out": out}, {"absmax": absmax})
     with torch.cuda.device(codes.device):
         st = load_library().dt8_dequantize_blockwise(
             _dev_tensor(codes, torch.uint8, "codes"), _dev_tensor(absmax, torch.float32, "absmax"), n,
@@ -216,6 +254,8 @@ def dt8_dequantize_blockwise(codes: torch.Tensor, absmax: torch.Tensor, block_si
 
 def dt8_sgd_step(p, g, m_codes, m_absmax, lr, momentum, weight_decay, step, block_size=2048,
                  stream=None) -> None:
+    _check_layout("dt8_sgd_step", p.numel(), block_size, p.device, {"g": g, "m_codes": m_codes},
+                  {"m_absmax": m_absmax})
     gp, gd = _grad_ptr(g)
     with torch.cuda.device(p.device):
         st = load_library().dt8_sgd_step(
@@ -227,6 +267,9 @@ def dt8_sgd_step(p, g, m_codes, m_absmax, lr, momentum, weight_decay, step, bloc
 
 def dt8_adam_step(p, g, m_codes, m_absmax, r_codes, r_absmax, lr, beta1, beta2, eps, weight_decay,
                   step, block_size=2048, flags=DEFAULT_ADAM_FLAGS, stream=None) -> None:
+    _check_layout("dt8_adam_step", p.numel(), block_size, p.device,
+                  {"g": g, "m_codes": m_codes, "r_codes": r_codes},
+                  {"m_absmax": m_absmax, "r_absmax": r_absmax})
     gp, gd = _grad_ptr(g)
     with torch.cuda.device(p.device):
         st = load_library().dt8_adam_step(
@@ -248,6 +291,25 @@ class _PtrList:
         return ctypes.cast(self.arr, ctypes.c_void_p)
 
 
+def _check_list_layout(where, block_size, ps, gs, m_codes, m_absmax, r_codes=None, r_absmax=None):
+    lists = {"g": gs, "m_codes": m_codes, "m_absmax": m_absmax}
+    if r_codes is not None:
+        lists["r_codes"], lists["r_absmax"] = r_codes, r_absmax
+    for name, lst in lists.items():
+        if len(lst) != len(ps):
+            raise ValueError(f"{where}: {name} lists {len(lst)} tensors, expected {len(ps)}")
+    dev = ps[0].device if len(ps) else None
+    for i, p in enumerate(ps):
+        by_el = {f"g[{i}]": gs[i], f"m_codes[{i}]": m_codes[i]}
+        by_bl = {f"m_absmax[{i}]": m_absmax[i]}
+        if r_codes is not None:
+            by_el[f"r_codes[{i}]"] = r_codes[i]
+            by_bl[f"r_absmax[{i}]"] = r_absmax[i]
+        if p.device != dev:
+            raise ValueError(f"{where}: p[{i}] is on {p.device}, expected {dev}")
+        _check_layout(where, p.numel(), block_size, dev, by_el, by_bl)
+
+
 def _multi_common(ps, gs):
     if len(ps) == 0:
         return None, None, None, None
@@ -263,6 +325,7 @@ def _multi_common(ps, gs):
 
 def dt8_sgd_step_multi(ps, gs, m_codes, m_absmax, lr, momentum, weight_decay, step, block_size=2048,
                        stream=None) -> None:
+    _check_list_layout("dt8_sgd_step_multi", block_size, ps, gs, m_codes, m_absmax)
     dev, gd, garr, narr = _multi_common(ps, gs)
     if dev is None:
         return
@@ -279,6 +342,7 @@ def dt8_sgd_step_multi(ps, gs, m_codes, m_absmax, lr, momentum, weight_decay, st
 
 def dt8_adam_step_multi(ps, gs, m_codes, m_absmax, r_codes, r_absmax, lr, beta1, beta2, eps,
                         weight_decay, step, block_size=2048, flags=DEFAULT_ADAM_FLAGS, stream=None) -> None:
+    _check_list_layout("dt8_adam_step_multi", block_size, ps, gs, m_codes, m_absmax, r_codes, r_absmax)
     dev, gd, garr, narr = _multi_common(ps, gs)
     if dev is None:
         return
@@ -316,8 +380,20 @@ class PreparedTensorList:
         self._ma = _PtrList(m_absmax, torch.float32, "m_absmax")
         self._rc = _PtrList(r_codes, torch.uint8, "r_codes") if r_codes is not None else None
         self._ra = _PtrList(r_absmax, torch.float32, "r_absmax") if r_absmax is not None else None
+        self._layout_checked = set()      # block sizes whose state sizes were verified
+
+    def _check_block_size(self, where: str, block_size: int) -> None:
+        """The sizes of the states depend on the block size, which arrives with the step: verify
+        them the first time a block size is used (the tensors cannot change size afterwards)."""
+        if block_size in self._layout_checked:
+            return
+        ps, gs, mc, ma, rc, ra = self._keep
+        _check_list_layout(where, block_size, ps, gs, mc, ma, rc if self._rc is not None else None,
+                           ra if self._ra is not None else None)
+        self._layout_checked.add(block_size)
 
     def sgd_step(self, lr, momentum, weight_decay, step, block_size=2048, stream=None) -> None:
+        self._check_block_size("PreparedTensorList.sgd_step", block_size)
         with torch.cuda.device(self.device):
             st = load_library().dt8_sgd_step_multi(
                 self.num, self._p.ptr, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
@@ -329,6 +405,7 @@ class PreparedTensorList:
                   flags=DEFAULT_ADAM_FLAGS, stream=None) -> None:
         if self._rc is None or self._ra is None:
             raise ValueError("this list was prepared without second-moment states")
+        self._check_block_size("PreparedTensorList.adam_step", block_size)
         with torch.cuda.device(self.device):
             st = load_library().dt8_adam_step_multi(
                 self.num, self._p.ptr, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
@@ -341,7 +418,7 @@ class PreparedTensorList:
 def shard_blocks(num_blocks_total: int, rank: int, world_size: int) -> range:
     """Contiguous range of whole quantization blocks owned by `rank`.
 
-    Blocks are independent (Section IV-B, "quantization applied independently to each block"),
+    Every block is quantized on its own (Section IV-B, "Tensor chunking"),
     so a tensor can be split across ranks on block boundaries with no exchange between them.
     The first `num_blocks_total % world_size` ranks own one extra block."""
     if not (0 <= rank < world_size):

@@ -4,6 +4,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <initializer_list>
 #include <mutex>
 
 #include "dt8.h"
@@ -117,37 +118,36 @@ int grid_for(int64_t blocks, int groups_per_cta, int sm_count) {
 
 // Values per thread and threads per CTA for each operation and block size.  A group (B / VPT
 // threads) is at least one warp, and the groups tile the CTA.
-#ifndef DT8_ADAM_VPT
-#define DT8_ADAM_VPT 16
-#endif
-#ifndef DT8_ADAM_THREADS
-#define DT8_ADAM_THREADS 512
-#endif
-#ifndef DT8_SGD_VPT
-#define DT8_SGD_VPT 16
-#endif
-#ifndef DT8_SGD_THREADS
-#define DT8_SGD_THREADS 512
-#endif
-#ifndef DT8_QUANT_VPT
-#define DT8_QUANT_VPT 16
-#endif
-#ifndef DT8_QUANT_THREADS
-#define DT8_QUANT_THREADS 1024
-#endif
 template <int B, int VPT_WANTED, int THREADS_WANTED> struct GeometryOf {
   static constexpr int VPT = (B / VPT_WANTED >= 32) ? VPT_WANTED : B / 32;
   static constexpr int THREADS = (THREADS_WANTED % (B / VPT) == 0) ? THREADS_WANTED : (B / VPT);
   static_assert(VPT % 4 == 0 && THREADS <= kCtaThreads && THREADS % (B / VPT) == 0, "bad geometry");
 };
-// Small blocks are latency-bound rather than issue-bound (one warp owns a block): 768 threads
-// with 8 values each measured 1-5 % faster there than 512 x 16.
-template <int B> struct AdamGeometry : GeometryOf<B, DT8_ADAM_VPT, DT8_ADAM_THREADS> {};
+// The steps run 512 threads x 16 values.  Small blocks are latency-bound rather than issue-bound
+// (one warp owns a block): 768 threads with 8 values each measured 1-5 % faster there.
+template <int B> struct AdamGeometry : GeometryOf<B, 16, 512> {};
 template <> struct AdamGeometry<256> : GeometryOf<256, 8, 768> {};
 template <> struct AdamGeometry<512> : GeometryOf<512, 8, 768> {};
-template <int B> struct SgdGeometry : GeometryOf<B, DT8_SGD_VPT, DT8_SGD_THREADS> {};
+template <int B> struct SgdGeometry : GeometryOf<B, 16, 512> {};
 template <> struct SgdGeometry<256> : GeometryOf<256, 8, 768> {};
-template <int B> using QuantGeometry = GeometryOf<B, DT8_QUANT_VPT, DT8_QUANT_THREADS>;
+template <int B> using QuantGeometry = GeometryOf<B, 16, 1024>;
+
+// Hyper-parameters are checked before anything is launched: non-finite values and decay rates
+// outside [0, 1) (1 - beta^step would be 0 or negative) are argument errors.
+bool finite_all(std::initializer_list<float> v) {
+  for (float x : v)
+    if (!std::isfinite(x)) return false;
+  return true;
+}
+
+bool adam_hyper_ok(float lr, float beta1, float beta2, float eps, float wd) {
+  return finite_all({lr, beta1, beta2, eps, wd}) && beta1 >= 0.0f && beta1 < 1.0f && beta2 >= 0.0f &&
+         beta2 < 1.0f && eps >= 0.0f;
+}
+
+bool sgd_hyper_ok(float lr, float momentum, float wd) {
+  return finite_all({lr, momentum, wd}) && momentum >= 0.0f;
+}
 
 int check_tensor(const TensorDesc& d, int g_dtype, bool adam) {
   if (d.n < 0) return DT8_ERR_INVALID_ARG;
@@ -183,6 +183,7 @@ int dispatch_adam_mode(const Args& args, int64_t blocks, int mode, const AdamHyp
   switch (mode) {
     case kAdamWFast: return launch_adam<Args, B, GBF16, kAdamWFast>(args, blocks, h, em, di, s);
     case kAdamWIeee: return launch_adam<Args, B, GBF16, kAdamWIeee>(args, blocks, h, em, di, s);
+    case kAdamWSmall: return launch_adam<Args, B, GBF16, kAdamWSmall>(args, blocks, h, em, di, s);
     default: return launch_adam<Args, B, GBF16, kAdamL2>(args, blocks, h, em, di, s);
   }
 }
@@ -259,6 +260,34 @@ int launch_quantize(const float* x, int64_t n, uint8_t* codes, float* absmax, co
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
 
+// Correctly rounded binary32 reciprocal of a positive normal binary32 number, on the host.  The
+// binary64 quotient rounded to binary32 can be one unit off (double rounding), so its two
+// neighbours are compared as well: |d*y - 1| is exact in binary64 (a 48-bit product, then a
+// difference of nearby numbers) and smallest for the nearest y.
+float reciprocal_rn(float d) {
+  const double dd = static_cast<double>(d);
+  const float y0 = static_cast<float>(1.0 / dd);
+  float best = y0;
+  double best_err = std::fabs(dd * static_cast<double>(y0) - 1.0);
+  const float cand[2] = {std::nextafterf(y0, 0.0f), std::nextafterf(y0, INFINITY)};
+  for (float y : cand) {
+    const double err = std::fabs(dd * static_cast<double>(y) - 1.0);
+    if (err < best_err) {
+      best_err = err;
+      best = y;
+    }
+  }
+  return best;
+}
+
+ConstDivisor make_const_divisor(float d) {
+  ConstDivisor cd;
+  cd.d = d;
+  cd.usable = d >= kConstDivMinDivisor && d <= kConstDivMaxDivisor;
+  cd.rd = cd.usable ? reciprocal_rn(d) : 0.0f;
+  return cd;
+}
+
 AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float wd, int64_t step,
                           uint32_t flags) {
   AdamHyper h;
@@ -282,22 +311,28 @@ AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float w
   h.eps_scaled = static_cast<float>(static_cast<double>(eps) * root_bc2);
   h.inv_step = static_cast<float>(1.0 / ss);
   h.eps_over_step = static_cast<float>(static_cast<double>(eps) * root_bc2 / ss);
+  const ConstDivisor d1 = make_const_divisor(h.bc1), d2 = make_const_divisor(h.bc2);
+  h.rbc1 = d1.rd;
+  h.rbc2 = d2.rd;
+  h.const_div = (d1.usable && d2.usable) ? 1 : 0;
   return h;
 }
 
 // The single-instruction root and reciprocal flush subnormal numbers to zero; a flushed root
-// (below 1.1e-19) is invisible next to the scaled eps only while that is well above it.
-constexpr float kMinEpsForFastUpdate = 1e-12f;
+// (below 1.1e-19) is invisible next to the scaled eps only while that is well above it.  Below
+// that the forms that keep subnormals are used.
+constexpr float kMinEpsForFlushedRoot = 1e-12f;
 
 // Coupled decay makes the parameters an input of the states, so they must then be computed with
-// IEEE operations; without decay the two forms coincide and the fast parameter path applies.
+// IEEE operations; without decay the two forms coincide and the approximate parameter path applies.
 int adam_mode(uint32_t flags, const AdamHyper& h) {
   if (!(flags & DT8_ADAM_DECOUPLED_WD) && h.wd != 0.0f) return kAdamL2;
-  // the fast path also divides by the step size, so that must be a normal, moderate number
-  const bool fast = h.eps_scaled >= kMinEpsForFastUpdate && h.lr >= 1e-20f && h.lr <= 1e20f &&
-                    std::isfinite(h.inv_step) && std::isfinite(h.eps_over_step) &&
-                    h.eps_over_step >= 1e-30f;
-  return fast ? kAdamWFast : kAdamWIeee;
+  // the approximate paths divide by the step size, so that must be a normal, moderate number
+  const bool moderate = h.lr >= 1e-20f && h.lr <= 1e20f && std::isfinite(h.inv_step) &&
+                        std::isfinite(h.eps_over_step) && h.inv_step >= 1e-30f;
+  if (!moderate) return kAdamWIeee;
+  const bool flush_ok = h.eps_scaled >= kMinEpsForFlushedRoot && h.eps_over_step >= 1e-30f;
+  return flush_ok ? kAdamWFast : kAdamWSmall;
 }
 
 }  // namespace
@@ -383,6 +418,22 @@ int dt8_selfcheck_divide(const float* s, const float* N, int64_t n, float* out, 
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
 
+int dt8_selfcheck_divide_const(const float* s, float d, int64_t n, float* out, void* stream) {
+  if (n < 0) return DT8_ERR_INVALID_ARG;
+  if (n == 0) return DT8_OK;
+  if (!s || !out) return DT8_ERR_INVALID_ARG;
+  if (!aligned(s, 4) || !aligned(out, 4)) return DT8_ERR_ALIGNMENT;
+  DeviceInfo di;
+  EncMeta em;
+  int rc = ensure_device(&di, &em);
+  if (rc != DT8_OK) return rc;
+  const int64_t ctas = (n + 255) / 256;
+  const int grid = static_cast<int>(ctas < 8 * di.sm_count ? ctas : 8 * di.sm_count);
+  divide_const_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(s, make_const_divisor(d), out, n);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
 int dt8_quantize_blockwise(const float* x, int64_t n, int block_size, int is_signed, uint8_t* codes,
                            float* absmax, void* stream) {
   if (n < 0) return DT8_ERR_INVALID_ARG;
@@ -440,7 +491,7 @@ int dt8_sgd_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float* 
                  float lr, float momentum, float weight_decay, int64_t step, int block_size,
                  void* stream) {
   if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
-  if (step < 1) return DT8_ERR_INVALID_ARG;
+  if (step < 1 || !sgd_hyper_ok(lr, momentum, weight_decay)) return DT8_ERR_INVALID_ARG;
   if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
   SingleArgs a;
   a.t = TensorDesc{p, g, m_codes, m_absmax, nullptr, nullptr, n};
@@ -462,6 +513,7 @@ int dt8_adam_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float*
                   void* stream) {
   if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
   if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
+  if (!adam_hyper_ok(lr, beta1, beta2, eps, weight_decay)) return DT8_ERR_INVALID_ARG;
   if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
   SingleArgs a;
   a.t = TensorDesc{p, g, m_codes, m_absmax, r_codes, r_absmax, n};
@@ -485,7 +537,9 @@ namespace {
 
 // Shared front end of the two pointer-list entry points: validates every tensor first (so that a
 // bad entry means nothing was launched), then launches one kernel per kMaxTensorsPerLaunch
-// non-empty tensors.
+// non-empty tensors.  Every tensor that passed the checks fits a launch of its own, so after the
+// checks only the CUDA runtime can fail (DT8_ERR_CUDA), possibly after earlier launches of the
+// same call were queued.
 template <class Launch>
 int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtype,
               uint8_t* const* mc, float* const* ma, uint8_t* const* rc, float* const* ra,
@@ -499,7 +553,7 @@ int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtyp
     const TensorDesc d{p[i], g[i], mc[i], ma[i], adam ? rc[i] : nullptr, adam ? ra[i] : nullptr, n[i]};
     const int st = check_tensor(d, g_dtype, adam);
     if (st != DT8_OK) return st;
-    if ((n[i] + block_size - 1) / block_size > 0x3FFFFFFF) return DT8_ERR_UNSUPPORTED;
+    if ((n[i] + block_size - 1) / block_size > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
   }
   DeviceInfo di;
   EncMeta em;
@@ -514,10 +568,7 @@ int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtyp
     while (i < num_tensors && args.num < kMaxTensorsPerLaunch) {
       if (n[i] > 0) {
         const int64_t nb = (n[i] + block_size - 1) / block_size;
-        if (blocks + nb > kMaxBlocksPerLaunch) {
-          if (args.num == 0) return DT8_ERR_UNSUPPORTED;
-          break;
-        }
+        if (blocks + nb > kMaxBlocksPerLaunch) break;   // args.num > 0 here: nb alone fits
         args.t[args.num] = TensorDesc{p[i], g[i], mc[i], ma[i], adam ? rc[i] : nullptr,
                                       adam ? ra[i] : nullptr, n[i]};
         blocks += nb;
@@ -541,7 +592,7 @@ int dt8_sgd_step_multi(int num_tensors, float* const* p, const void* const* g, i
                        uint8_t* const* m_codes, float* const* m_absmax, const int64_t* n, float lr,
                        float momentum, float weight_decay, int64_t step, int block_size,
                        void* stream) {
-  if (step < 1) return DT8_ERR_INVALID_ARG;
+  if (step < 1 || !sgd_hyper_ok(lr, momentum, weight_decay)) return DT8_ERR_INVALID_ARG;
   const SgdHyper h{lr, momentum, weight_decay};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   return run_multi(num_tensors, p, g, g_dtype, m_codes, m_absmax, nullptr, nullptr, n, block_size,
@@ -556,6 +607,7 @@ int dt8_adam_step_multi(int num_tensors, float* const* p, const void* const* g, 
                         float eps, float weight_decay, int64_t step, int block_size, uint32_t flags,
                         void* stream) {
   if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
+  if (!adam_hyper_ok(lr, beta1, beta2, eps, weight_decay)) return DT8_ERR_INVALID_ARG;
   const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
   const int mode = adam_mode(flags, h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);

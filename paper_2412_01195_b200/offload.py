@@ -56,6 +56,11 @@ class StreamedAdam8bit:
         for t in (w, g, m_codes, m_absmax, r_codes, r_absmax):
             if t.is_cuda or not t.is_contiguous():
                 raise TypeError("host, contiguous tensors are required")
+        if g.dtype != self.sets[0]["g"].dtype:
+            raise TypeError("g: the gradient dtype this object was built for is required")
+        dt8._check_layout("StreamedAdam8bit.step", n, B, w.device,
+                          {"g": g, "m_codes": m_codes, "r_codes": r_codes},
+                          {"m_absmax": m_absmax, "r_absmax": r_absmax})
         cur = torch.cuda.current_stream(self.device)
         start = torch.cuda.Event()
         start.record(cur)

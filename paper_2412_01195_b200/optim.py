@@ -77,6 +77,15 @@ class _Optimizer8bit(torch.optim.Optimizer):
         for pid, p in zip(ids, params):
             for k, v in codes.get(pid, {}).items():
                 self.state[p][k] = v.detach().to(device=p.device, dtype=torch.uint8).clone()
+        # a state saved with another block size (or for another tensor) must not reach a kernel
+        for group in self.param_groups:
+            for p in group["params"]:
+                st = self.state.get(p, {})
+                if "m_codes" not in st:
+                    continue
+                by_el = {k: st[k] for k in ("m_codes", "r_codes") if k in st}
+                by_bl = {k: st[k] for k in ("m_absmax", "r_absmax") if k in st}
+                dt8._check_layout("load_state_dict", p.numel(), group["block_size"], p.device, by_el, by_bl)
         self._prepared.clear()
 
     def state_bytes(self) -> int:

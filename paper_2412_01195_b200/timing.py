@@ -188,6 +188,9 @@ def main():
         elif case == "adaml2":
             adam_case(report, dev, 1 << 28, f32, "adam fp32 grads, coupled decay (IEEE path) n=2^28",
                       flags=dt8.DT8_ADAM_BIAS_CORRECTION)
+        elif case == "adaml226":
+            adam_case(report, dev, 1 << 26, f32, "adam fp32 grads, coupled decay (IEEE path) n=2^26",
+                      flags=dt8.DT8_ADAM_BIAS_CORRECTION)
         elif case == "sgd":
             sgd_case(report, dev, 1 << 28, f32, "sgd fp32 grads n=2^28 B=2048")
         elif case == "sgd26":

@@ -179,6 +179,79 @@ def test_argument_checks_return_before_any_device_work(lib):
     assert adamm(0, None, None, None) == E.DT8_OK
 
 
+def test_hyper_parameters_are_validated_before_any_device_work(lib):
+    """Non-finite values, decay rates outside [0, 1), negative eps / momentum: argument errors."""
+    f = ctypes.c_float
+    buf = (ctypes.c_uint8 * 4096)()
+    base = ctypes.addressof(buf)
+    ok = ctypes.c_void_p(base + (-base) % 16)
+    E = dt8
+    adam = lambda lr=1e-3, b1=.9, b2=.999, eps=1e-8, wd=0.: lib.dt8_adam_step(
+        ok, ok, 0, ok, ok, ok, ok, 16, f(lr), f(b1), f(b2), f(eps), f(wd), 1, 2048, 3, None)
+    for kw in (dict(lr=float("nan")), dict(lr=float("inf")), dict(b1=1.0), dict(b2=1.0), dict(b1=-0.1),
+               dict(b2=1.5), dict(eps=-1e-8), dict(eps=float("nan")), dict(wd=float("inf"))):
+        assert adam(**kw) == E.DT8_ERR_INVALID_ARG, kw
+    sgd = lambda lr=.1, mom=.9, wd=0.: lib.dt8_sgd_step(ok, ok, 0, ok, ok, 16, f(lr), f(mom), f(wd), 1, 2048, None)
+    for kw in (dict(lr=float("nan")), dict(mom=float("inf")), dict(mom=-0.5), dict(wd=float("nan"))):
+        assert sgd(**kw) == E.DT8_ERR_INVALID_ARG, kw
+    arr = (ctypes.c_void_p * 1)(ok.value)
+    ns = (ctypes.c_int64 * 1)(16)
+    ap, nsp = ctypes.cast(arr, ctypes.c_void_p), ctypes.cast(ns, ctypes.c_void_p)
+    assert lib.dt8_adam_step_multi(1, ap, ap, 0, ap, ap, ap, ap, nsp, f(1e-3), f(1.0), f(.999), f(1e-8),
+                                   f(0), 1, 2048, 3, None) == E.DT8_ERR_INVALID_ARG
+    assert lib.dt8_sgd_step_multi(1, ap, ap, 0, ap, ap, nsp, f(float("nan")), f(.9), f(0), 1, 2048,
+                                  None) == E.DT8_ERR_INVALID_ARG
+    # the pointer-list forms accept as many blocks per tensor as the single-tensor forms do
+    big = (ctypes.c_int64 * 1)((0x7FFF0000 + 1) * 256)
+    assert lib.dt8_sgd_step_multi(1, ap, ap, 0, ap, ap, ctypes.cast(big, ctypes.c_void_p), f(.1), f(.9),
+                                  f(0), 1, 256, None) == E.DT8_ERR_UNSUPPORTED
+    assert lib.dt8_sgd_step(ok, ok, 0, ok, ok, (0x7FFF0000 + 1) * 256, f(.1), f(.9), f(0), 1, 256,
+                            None) == E.DT8_ERR_UNSUPPORTED
+
+
+class _NoLaunch:
+    """Stands where the loaded library would be: any attempt to call into it fails the test."""
+
+    def __getattr__(self, name):
+        raise AssertionError(f"the binding reached the library ({name}) with inconsistent sizes")
+
+
+def test_binding_refuses_inconsistent_sizes_before_the_call(monkeypatch):
+    """A state built for one block size stepped with another, a gradient of another length, a
+    state list of another length: the binding raises ValueError and never reaches the library
+    (the C ABI takes n and block_size on trust and would write past the absmax array)."""
+    import torch
+    monkeypatch.setattr(dt8, "_lib", _NoLaunch())
+    n, B = 8 * 2048, 2048
+    p, g = torch.zeros(n), torch.zeros(n)
+    codes = torch.zeros(n, dtype=torch.uint8)
+    am = torch.zeros(n // B)
+    hp = (1e-3, 0.9, 0.999, 1e-8, 0.0, 1)
+    with pytest.raises(ValueError, match="block maxima"):
+        dt8.dt8_adam_step(p, g, codes, am, codes, am, *hp, 256)           # state built for B = 2048
+    with pytest.raises(ValueError, match="g holds"):
+        dt8.dt8_adam_step(p, g[:-1], codes, am, codes, am, *hp, B)
+    with pytest.raises(ValueError, match="r_codes holds"):
+        dt8.dt8_adam_step(p, g, codes, am, codes[:5], am, *hp, B)
+    with pytest.raises(ValueError, match="block_size"):
+        dt8.dt8_adam_step(p, g, codes, am, codes, am, *hp, 1000)
+    with pytest.raises(ValueError, match="block maxima"):
+        dt8.dt8_sgd_step(p, g, codes, am[:-1], 0.1, 0.9, 0.0, 1, B)
+    with pytest.raises(ValueError, match="block maxima"):
+        dt8.dt8_quantize_blockwise(p, 256, True, codes, am)
+    with pytest.raises(ValueError, match="out holds"):
+        dt8.dt8_dequantize_blockwise(codes, am, B, True, torch.zeros(n - 1))
+    with pytest.raises(ValueError, match="lists 1 tensors"):
+        dt8.dt8_adam_step_multi([p, p], [g, g], [codes, codes], [am, am], [codes], [am, am], *hp, B)
+    with pytest.raises(ValueError, match=r"m_absmax\[1\]"):
+        dt8.dt8_sgd_step_multi([p, p], [g, g], [codes, codes], [am, am[:3]], 0.1, 0.9, 0.0, 1, B)
+    with pytest.raises(ValueError, match="is on"):
+        dt8._check_layout("x", n, B, torch.device("cuda", 0), {"g": g}, {})
+    # consistent sizes pass the layout check and stop at the next one (these are host tensors)
+    with pytest.raises(TypeError, match="CUDA tensor"):
+        dt8.dt8_adam_step(p, g, codes, am, codes, am, *hp, B)
+
+
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(dt8, "_lib", None)
     monkeypatch.setattr(dt8, "_LIB_PATH", str(tmp_path / "nope.so"))

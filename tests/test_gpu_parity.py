@@ -216,7 +216,9 @@ def test_adam_variants(flags):
 
 def test_adam_literal_equation_without_decay_and_tiny_eps():
     """Eq. adam exactly as printed (no bias correction, no decay) takes the fast parameter path
-    (1e-6); an eps too small for that path takes IEEE operations (bit-exact parameters)."""
+    (1e-6); an eps too small to hide a flushed subnormal root takes the forms of the root and
+    reciprocal that keep subnormals (1e-6 as well); a learning rate outside the range of the
+    approximate paths takes IEEE operations (bit-exact parameters)."""
     n, B = 21 * 2048 + 77, 2048
     hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
     st = AdamState(synth.normal(n, 0.02, 610), B)
@@ -226,7 +228,15 @@ def test_adam_literal_equation_without_decay_and_tiny_eps():
     hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-20, weight_decay=0.01)
     st = AdamState(synth.normal(n, 0.02, 611), B)
     for t in range(1, 6):
-        st.step(synth.fresh_grad(n, 45, t), t, hp)
+        g = synth.fresh_grad(n, 45, t)
+        g[5 * B:6 * B] *= 1e-18                      # second moments down in the subnormal range
+        g[6 * B:7 * B] = 0.0
+        st.step(g, t, hp)
+    st.check()
+    hp = dict(lr=1e-25, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    st = AdamState(synth.normal(n, 0.02, 612), B)
+    for t in range(1, 6):
+        st.step(synth.fresh_grad(n, 46, t), t, hp)
     st.check(exact_params=True)
 
 
