@@ -32,7 +32,8 @@
  *     block_size 2048), in the single-tensor and the pointer-list forms alike, else
  *     DT8_ERR_UNSUPPORTED.
  *   - Alignment: fp32 tensors 16 bytes, bf16 tensors 8 bytes, code arrays 4 bytes, absmax arrays
- *     4 bytes, at each tensor's base; else DT8_ERR_ALIGNMENT.
+ *     4 bytes, at each tensor's base; else DT8_ERR_ALIGNMENT.  Nothing more is assumed: a code
+ *     array at a 4-byte-only offset or a parameter tensor at a 16-byte-only offset is fine.
  *   - n == 0 (or num_tensors == 0) is a successful no-op.  n < 0, a NULL tensor pointer with
  *     n > 0, step < 1, or an unknown dtype / flag gives DT8_ERR_INVALID_ARG.  So do non-finite
  *     hyper-parameters, beta1 or beta2 outside [0, 1), a negative eps and a negative momentum.
@@ -62,7 +63,7 @@ typedef enum {
   DT8_ERR_CUDA = 4
 } dt8_status;
 
-/* Gradient element type. */
+/* Element type of gradients and, in the _ex entry points, of parameters. */
 typedef enum { DT8_F32 = 0, DT8_BF16 = 1 } dt8_dtype;
 
 /* Flags of dt8_adam_step.  The default used by the Python binding is both bits set (AdamW with
@@ -178,14 +179,35 @@ int dt8_sgd_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *
  *     m' is re-quantized with the signed table, r' with the unsigned table.
  * The parameter update uses the 32-bit m', r' before they are quantized.  With decoupled decay, or
  * with weight_decay == 0, the parameter update is evaluated with a single-instruction reciprocal
- * and square root (relative error ~2e-7 of the update term); with coupled decay, where p feeds the
- * states, and whenever eps*sqrt(bc2) < 1e-12 (a flushed subnormal root would show), it is
- * evaluated with IEEE operations and is bit-reproducible against a plain binary32 evaluation.
+ * and square root (relative error ~2e-7 of the update term; when eps*sqrt(bc2) < 1e-12 the forms
+ * of these instructions that keep subnormal numbers are used, so that a tiny second moment is not
+ * flushed to zero).  With coupled decay, where p feeds the states, and for a learning rate outside
+ * 1e-20 .. 1e20, it is evaluated with IEEE operations and is bit-reproducible against a plain
+ * binary32 evaluation.
  */
 int dt8_adam_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
                   uint8_t *r_codes, float *r_absmax, int64_t n, float lr, float beta1, float beta2,
                   float eps, float weight_decay, int64_t step, int block_size, uint32_t flags,
                   void *stream);
+
+/*
+ * The same two steps for parameters of either element type (p_dtype: DT8_F32 or DT8_BF16).
+ * The paper keeps parameters in 32-bit floating point (Section II); bfloat16 parameters without a
+ * 32-bit copy are a variant of this library: the stored parameter is widened exactly, the update
+ * of Eq. sgd / Eq. adam is evaluated in binary32 exactly as for binary32 parameters, and the
+ * result is rounded once, to nearest even, when it is stored.  States and their arithmetic do
+ * not change.  bfloat16 parameters need 8-byte alignment.  dt8_sgd_step(p, ...) is
+ * dt8_sgd_step_ex(p, DT8_F32, ...), and likewise for Adam.
+ *   p   device, float[n] or bf16[n] per p_dtype, updated in place
+ */
+int dt8_sgd_step_ex(void *p, int p_dtype, const void *g, int g_dtype, uint8_t *m_codes,
+                    float *m_absmax, int64_t n, float lr, float momentum, float weight_decay,
+                    int64_t step, int block_size, void *stream);
+
+int dt8_adam_step_ex(void *p, int p_dtype, const void *g, int g_dtype, uint8_t *m_codes,
+                     float *m_absmax, uint8_t *r_codes, float *r_absmax, int64_t n, float lr,
+                     float beta1, float beta2, float eps, float weight_decay, int64_t step,
+                     int block_size, uint32_t flags, void *stream);
 
 /*
  * Pointer-list forms: the same step applied to num_tensors tensors in one kernel launch per 256
@@ -206,6 +228,19 @@ int dt8_adam_step_multi(int num_tensors, float *const *p, const void *const *g, 
                         float *const *r_absmax, const int64_t *n, float lr, float beta1,
                         float beta2, float eps, float weight_decay, int64_t step, int block_size,
                         uint32_t flags, void *stream);
+
+/* Pointer-list forms for parameters of either element type (all parameters of a call share
+ * p_dtype); otherwise as above. */
+int dt8_sgd_step_multi_ex(int num_tensors, void *const *p, int p_dtype, const void *const *g,
+                          int g_dtype, uint8_t *const *m_codes, float *const *m_absmax,
+                          const int64_t *n, float lr, float momentum, float weight_decay,
+                          int64_t step, int block_size, void *stream);
+
+int dt8_adam_step_multi_ex(int num_tensors, void *const *p, int p_dtype, const void *const *g,
+                           int g_dtype, uint8_t *const *m_codes, float *const *m_absmax,
+                           uint8_t *const *r_codes, float *const *r_absmax, const int64_t *n,
+                           float lr, float beta1, float beta2, float eps, float weight_decay,
+                           int64_t step, int block_size, uint32_t flags, void *stream);
 
 #ifdef __cplusplus
 }

@@ -40,6 +40,7 @@ EXPORTS = (
     "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_init", "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step",
     "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
+    "dt8_sgd_step_ex", "dt8_adam_step_ex", "dt8_sgd_step_multi_ex", "dt8_adam_step_multi_ex",
 )
 
 
@@ -86,6 +87,12 @@ def load_library() -> ctypes.CDLL:
     lib.dt8_sgd_step_multi.argtypes = [i32, vp, vp, i32, vp, vp, vp, f32, f32, f32, i64, i32, vp]
     lib.dt8_adam_step_multi.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, vp, f32, f32, f32, f32, f32,
                                         i64, i32, u32, vp]
+    lib.dt8_sgd_step_ex.argtypes = [vp, i32, vp, i32, vp, vp, i64, f32, f32, f32, i64, i32, vp]
+    lib.dt8_adam_step_ex.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64,
+                                     i32, u32, vp]
+    lib.dt8_sgd_step_multi_ex.argtypes = [i32, vp, i32, vp, i32, vp, vp, vp, f32, f32, f32, i64, i32, vp]
+    lib.dt8_adam_step_multi_ex.argtypes = [i32, vp, i32, vp, i32, vp, vp, vp, vp, vp, f32, f32, f32, f32,
+                                           f32, i64, i32, u32, vp]
     for name in EXPORTS:
         getattr(lib, name).restype = getattr(lib, name).restype or i32
     _lib = lib
@@ -131,14 +138,15 @@ def _check_layout(where: str, n: int, block_size: int, device, by_elements: dict
             raise ValueError(f"{where}: {name} is on {t.device}, expected {device}")
 
 
-def _grad_ptr(g: torch.Tensor):
+def _grad_ptr(g: torch.Tensor, name: str = "g"):
+    """(device pointer, dt8_dtype) of a gradient or parameter tensor: float32 or bfloat16."""
     if not (isinstance(g, torch.Tensor) and g.is_cuda and g.is_contiguous()):
-        raise TypeError("g: need a contiguous CUDA tensor")
+        raise TypeError(f"{name}: need a contiguous CUDA tensor")
     if g.dtype == torch.float32:
         return g.data_ptr(), DT8_F32
     if g.dtype == torch.bfloat16:
         return g.data_ptr(), DT8_BF16
-    raise TypeError("g: float32 or bfloat16")
+    raise TypeError(f"{name}: float32 or bfloat16")
 
 
 # -----------------------------------------------------------------------------------------------
@@ -257,9 +265,10 @@ def dt8_sgd_step(p, g, m_codes, m_absmax, lr, momentum, weight_decay, step, bloc
     _check_layout("dt8_sgd_step", p.numel(), block_size, p.device, {"g": g, "m_codes": m_codes},
                   {"m_absmax": m_absmax})
     gp, gd = _grad_ptr(g)
+    pp, pd = _grad_ptr(p, "p")
     with torch.cuda.device(p.device):
-        st = load_library().dt8_sgd_step(
-            _dev_tensor(p, torch.float32, "p"), gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
+        st = load_library().dt8_sgd_step_ex(
+            pp, pd, gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
             _dev_tensor(m_absmax, torch.float32, "m_absmax"), p.numel(), lr, momentum, weight_decay,
             step, block_size, _stream_ptr(stream, p.device))
     _check(st, "dt8_sgd_step")
@@ -271,9 +280,10 @@ def dt8_adam_step(p, g, m_codes, m_absmax, r_codes, r_absmax, lr, beta1, beta2, 
                   {"g": g, "m_codes": m_codes, "r_codes": r_codes},
                   {"m_absmax": m_absmax, "r_absmax": r_absmax})
     gp, gd = _grad_ptr(g)
+    pp, pd = _grad_ptr(p, "p")
     with torch.cuda.device(p.device):
-        st = load_library().dt8_adam_step(
-            _dev_tensor(p, torch.float32, "p"), gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
+        st = load_library().dt8_adam_step_ex(
+            pp, pd, gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
             _dev_tensor(m_absmax, torch.float32, "m_absmax"), _dev_tensor(r_codes, torch.uint8, "r_codes"),
             _dev_tensor(r_absmax, torch.float32, "r_absmax"), p.numel(), lr, beta1, beta2, eps,
             weight_decay, step, block_size, flags, _stream_ptr(stream, p.device))
@@ -310,17 +320,28 @@ def _check_list_layout(where, block_size, ps, gs, m_codes, m_absmax, r_codes=Non
         _check_layout(where, p.numel(), block_size, dev, by_el, by_bl)
 
 
+class _TypedPtrList:
+    """Host array of device pointers of tensors that share one of the two element types."""
+
+    def __init__(self, tensors: Sequence[torch.Tensor], name: str):
+        dt = tensors[0].dtype
+        if any(t.dtype != dt for t in tensors):
+            raise TypeError(f"all {name} tensors of one call share a dtype")
+        self.dtype = _grad_ptr(tensors[0], name)[1]
+        self.arr = (ctypes.c_void_p * len(tensors))(*[_grad_ptr(t, name)[0] for t in tensors])
+
+    @property
+    def ptr(self):
+        return ctypes.cast(self.arr, ctypes.c_void_p)
+
+
 def _multi_common(ps, gs):
     if len(ps) == 0:
         return None, None, None, None
     dev = ps[0].device
-    gdt = gs[0].dtype
-    if any(g.dtype != gdt for g in gs):
-        raise TypeError("all gradients of one call share a dtype")
-    _, gd = _grad_ptr(gs[0])
-    garr = (ctypes.c_void_p * len(gs))(*[_grad_ptr(g)[0] for g in gs])
+    g = _TypedPtrList(gs, "g")
     narr = (ctypes.c_int64 * len(ps))(*[p.numel() for p in ps])
-    return dev, gd, garr, narr
+    return dev, g.dtype, g.arr, narr
 
 
 def dt8_sgd_step_multi(ps, gs, m_codes, m_absmax, lr, momentum, weight_decay, step, block_size=2048,
@@ -329,12 +350,12 @@ def dt8_sgd_step_multi(ps, gs, m_codes, m_absmax, lr, momentum, weight_decay, st
     dev, gd, garr, narr = _multi_common(ps, gs)
     if dev is None:
         return
-    pl = _PtrList(ps, torch.float32, "p")
+    pl = _TypedPtrList(ps, "p")
     mc = _PtrList(m_codes, torch.uint8, "m_codes")
     ma = _PtrList(m_absmax, torch.float32, "m_absmax")
     with torch.cuda.device(dev):
-        st = load_library().dt8_sgd_step_multi(
-            len(ps), pl.ptr, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr,
+        st = load_library().dt8_sgd_step_multi_ex(
+            len(ps), pl.ptr, pl.dtype, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr,
             ctypes.cast(narr, ctypes.c_void_p), lr, momentum, weight_decay, step, block_size,
             _stream_ptr(stream, dev))
     _check(st, "dt8_sgd_step_multi")
@@ -346,14 +367,14 @@ def dt8_adam_step_multi(ps, gs, m_codes, m_absmax, r_codes, r_absmax, lr, beta1,
     dev, gd, garr, narr = _multi_common(ps, gs)
     if dev is None:
         return
-    pl = _PtrList(ps, torch.float32, "p")
+    pl = _TypedPtrList(ps, "p")
     mc = _PtrList(m_codes, torch.uint8, "m_codes")
     ma = _PtrList(m_absmax, torch.float32, "m_absmax")
     rc = _PtrList(r_codes, torch.uint8, "r_codes")
     ra = _PtrList(r_absmax, torch.float32, "r_absmax")
     with torch.cuda.device(dev):
-        st = load_library().dt8_adam_step_multi(
-            len(ps), pl.ptr, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr, rc.ptr, ra.ptr,
+        st = load_library().dt8_adam_step_multi_ex(
+            len(ps), pl.ptr, pl.dtype, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr, rc.ptr, ra.ptr,
             ctypes.cast(narr, ctypes.c_void_p), lr, beta1, beta2, eps, weight_decay, step, block_size,
             flags, _stream_ptr(stream, dev))
     _check(st, "dt8_adam_step_multi")
@@ -375,7 +396,7 @@ class PreparedTensorList:
                       list(r_codes or []), list(r_absmax or []))
         self.device, self.g_dtype, self._g, self._n = _multi_common(ps, gs)
         self.num = len(ps)
-        self._p = _PtrList(ps, torch.float32, "p")
+        self._p = _TypedPtrList(ps, "p")
         self._mc = _PtrList(m_codes, torch.uint8, "m_codes")
         self._ma = _PtrList(m_absmax, torch.float32, "m_absmax")
         self._rc = _PtrList(r_codes, torch.uint8, "r_codes") if r_codes is not None else None
@@ -395,8 +416,8 @@ class PreparedTensorList:
     def sgd_step(self, lr, momentum, weight_decay, step, block_size=2048, stream=None) -> None:
         self._check_block_size("PreparedTensorList.sgd_step", block_size)
         with torch.cuda.device(self.device):
-            st = load_library().dt8_sgd_step_multi(
-                self.num, self._p.ptr, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
+            st = load_library().dt8_sgd_step_multi_ex(
+                self.num, self._p.ptr, self._p.dtype, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
                 self._mc.ptr, self._ma.ptr, ctypes.cast(self._n, ctypes.c_void_p), lr, momentum,
                 weight_decay, step, block_size, _stream_ptr(stream, self.device))
         _check(st, "dt8_sgd_step_multi")
@@ -407,8 +428,8 @@ class PreparedTensorList:
             raise ValueError("this list was prepared without second-moment states")
         self._check_block_size("PreparedTensorList.adam_step", block_size)
         with torch.cuda.device(self.device):
-            st = load_library().dt8_adam_step_multi(
-                self.num, self._p.ptr, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
+            st = load_library().dt8_adam_step_multi_ex(
+                self.num, self._p.ptr, self._p.dtype, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
                 self._mc.ptr, self._ma.ptr, self._rc.ptr, self._ra.ptr,
                 ctypes.cast(self._n, ctypes.c_void_p), lr, beta1, beta2, eps, weight_decay, step,
                 block_size, flags, _stream_ptr(stream, self.device))

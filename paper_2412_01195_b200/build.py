@@ -1,18 +1,31 @@
-"""Builds libdt8.so (the CUDA library behind the C ABI) in-tree with nvcc for sm_100a."""
+"""Builds libdt8.so (the CUDA library behind the C ABI) in-tree with nvcc for sm_100a.
+
+The kernels are instantiated in several translation units, compiled in parallel into
+``csrc/_build/*.o`` and linked into one shared library."""
 from __future__ import annotations
 
+import glob
 import os
 import shutil
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
+OBJ_DIR = os.path.join(CSRC, "_build")
 LIB = os.path.join(HERE, "libdt8.so")
-SOURCES = [os.path.join(CSRC, "dt8.cu"), os.path.join(CSRC, "dt8_tables.cpp")]
-HEADERS = [os.path.join(CSRC, "dt8_kernels.cuh"), os.path.join(CSRC, "dt8_tables.h"),
-           os.path.join(ROOT, "include", "dt8.h")]
+INCLUDE = os.path.join(ROOT, "include")
+
+
+def sources():
+    return sorted(glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cpp")))
+
+
+def headers():
+    return sorted(glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) +
+                  glob.glob(os.path.join(INCLUDE, "*.h")))
 
 
 def find_nvcc() -> str:
@@ -26,19 +39,36 @@ def is_stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(f) > t for f in SOURCES + HEADERS)
+    return any(os.path.getmtime(f) > t for f in sources() + headers())
+
+
+def _compile_one(nvcc: str, src: str, verbose: bool) -> str:
+    obj = os.path.join(OBJ_DIR, os.path.splitext(os.path.basename(src))[0] + ".o")
+    newest_dep = max(os.path.getmtime(f) for f in [src] + headers())
+    if os.path.exists(obj) and os.path.getmtime(obj) >= newest_dep:
+        return obj
+    cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+           "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC, "-c", src, "-o", obj + ".tmp"]
+    if verbose:
+        cmd += ["-Xptxas", "-v"]
+    subprocess.run(cmd, check=True)
+    os.replace(obj + ".tmp", obj)
+    return obj
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB
+    nvcc = find_nvcc()
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    if force:
+        for f in glob.glob(os.path.join(OBJ_DIR, "*.o")):
+            os.remove(f)
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        objs = list(pool.map(lambda s: _compile_one(nvcc, s, verbose), sources()))
     tmp = LIB + ".%d.tmp" % os.getpid()
-    cmd = [find_nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a",
-           "-lineinfo", "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"),
-           "-I", CSRC, "-o", tmp] + SOURCES
-    if verbose:
-        cmd += ["-Xptxas", "-v"]
-    subprocess.run(cmd, check=True)
+    subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs,
+                   check=True)
     os.replace(tmp, LIB)
     return LIB
 

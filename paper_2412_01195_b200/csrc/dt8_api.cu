@@ -1,4 +1,5 @@
-// C ABI of the dt8 library: argument checks, table upload, kernel selection and launch.
+// C ABI of the dt8 library: argument checks, table upload and the calls into the launchers of
+// the other translation units.
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -8,37 +9,78 @@
 #include <mutex>
 
 #include "dt8.h"
-#include "dt8_kernels.cuh"
+#include "dt8_launch.h"
 
 namespace dt8 {
-namespace {
 
+namespace {
 thread_local int tl_last_cuda_error = 0;
+}  // namespace
 
 int cuda_fail(cudaError_t e) {
   tl_last_cuda_error = static_cast<int>(e);
   return DT8_ERR_CUDA;
 }
 
-constexpr int kMaxDevices = 64;
+namespace {
 
-struct DeviceInfo {
-  int device = -1;
-  int sm_count = 0;
-};
+// The constant tables, one copy per device (this translation unit owns them; the kernels of the
+// other units receive the address).
+__device__ DeviceTables g_tables;
+
+// Shared-memory address at which a kernel's dynamic shared memory starts, written by
+// smem_start_probe and read back once per device.
+__device__ uint32_t g_smem_start;
+
+__global__ void smem_start_probe() {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  if (threadIdx.x == 0) g_smem_start = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw));
+}
+
+// Diagnostic: s_i / d by the constant-divisor routine of the IEEE Adam update.
+__global__ void __launch_bounds__(256)
+divide_const_kernel(const float* __restrict__ s, ConstDivisor cd, float* __restrict__ out, int64_t n) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+  {
+    const float a = fabsf(s[i]);
+    const bool fast = cd.usable && a >= kConstDivMinDividend && a <= kConstDivMaxDividend;
+    out[i] = fast ? cd.div<true>(s[i]) : cd.div<false>(s[i]);
+  }
+}
+
+// Diagnostic: the normalising division of the encoder applied to arbitrary operand pairs.
+__global__ void __launch_bounds__(256)
+divide_kernel(const float* __restrict__ s, const float* __restrict__ N, float* __restrict__ out,
+              int64_t n) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const Normaliser nz(N[i]);
+    out[i] = nz.fast ? nz.div<true>(s[i]) : nz.div<false>(s[i]);
+  }
+}
+
+
+constexpr int kMaxDevices = 64;
 
 std::mutex g_init_mutex;
 std::atomic<bool> g_uploaded[kMaxDevices];
 int g_sm_count[kMaxDevices];
+const DeviceTables* g_tables_addr[kMaxDevices];
 
-// Makes sure the current device holds the constant tables; returns the device's SM count.
-int ensure_device(DeviceInfo* info, EncMeta* em) {
+// Makes sure the current device holds the constant tables and fills the launch context.
+int ensure_device(LaunchCtx* ctx, void* stream) {
   const Tables* ht = host_tables();
   if (!ht) return DT8_ERR_UNSUPPORTED;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
   if (dev < 0 || dev >= kMaxDevices) return DT8_ERR_UNSUPPORTED;
+  EncMeta em;
+  em.s_first = ht->enc_signed.first_key;
+  em.u_first = ht->enc_unsigned.first_key;
+  em.s_n = ht->enc_signed.num_entries;
+  em.u_n = ht->enc_unsigned.num_entries;
   if (!g_uploaded[dev].load(std::memory_order_acquire)) {
     std::lock_guard<std::mutex> lock(g_init_mutex);
     if (!g_uploaded[dev].load(std::memory_order_relaxed)) {
@@ -51,15 +93,13 @@ int ensure_device(DeviceInfo* info, EncMeta* em) {
       std::memcpy(staging.enc_u, ht->enc_unsigned.entries, sizeof(uint32_t) * ht->enc_unsigned.num_entries);
       e = cudaMemcpyToSymbol(g_tables, &staging, sizeof(staging));
       if (e != cudaSuccess) return cuda_fail(e);
+      void* addr = nullptr;
+      e = cudaGetSymbolAddress(&addr, g_tables);
+      if (e != cudaSuccess) return cuda_fail(e);
       // The kernels address their shared-memory tables absolutely: check once that this build's
       // tables fit the layout and that dynamic shared memory starts low enough on this device.
-      EncMeta probe_em;
-      probe_em.s_first = ht->enc_signed.first_key;
-      probe_em.u_first = ht->enc_unsigned.first_key;
-      probe_em.s_n = ht->enc_signed.num_entries;
-      probe_em.u_n = ht->enc_unsigned.num_entries;
-      if (!layout_ok(probe_em)) return DT8_ERR_UNSUPPORTED;
-      const int probe_smem = static_cast<int>(smem_bytes(probe_em, true, true, true, true));
+      if (!layout_ok(em)) return DT8_ERR_UNSUPPORTED;
+      const int probe_smem = static_cast<int>(smem_bytes(em, true, true, true, true));
       e = cudaFuncSetAttribute(smem_start_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem);
       if (e != cudaSuccess) return cuda_fail(e);
       smem_start_probe<<<1, 32, probe_smem>>>();
@@ -73,64 +113,23 @@ int ensure_device(DeviceInfo* info, EncMeta* em) {
       e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
       if (e != cudaSuccess) return cuda_fail(e);
       g_sm_count[dev] = sms;
+      g_tables_addr[dev] = static_cast<const DeviceTables*>(addr);
       g_uploaded[dev].store(true, std::memory_order_release);
     }
   }
-  info->device = dev;
-  info->sm_count = g_sm_count[dev];
-  em->s_first = ht->enc_signed.first_key;
-  em->u_first = ht->enc_unsigned.first_key;
-  em->s_n = ht->enc_signed.num_entries;
-  em->u_n = ht->enc_unsigned.num_entries;
+  ctx->device = dev;
+  ctx->sm_count = g_sm_count[dev];
+  ctx->em = em;
+  ctx->tables = g_tables_addr[dev];
+  ctx->stream = static_cast<cudaStream_t>(stream);
   return DT8_OK;
-}
-
-// Opt a kernel in to its dynamic shared memory size, once per device.  `done` is the caller's
-// per-kernel flag word (kernels of different template arguments can share a pointer type, so the
-// flag cannot live in this function).
-template <class K>
-cudaError_t allow_smem(std::atomic<uint64_t>& done, K kernel, int device, size_t bytes) {
-  const uint64_t bit = 1ull << device;
-  if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(bytes));
-  if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_release);
-  return e;
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-// The kernels index quantization blocks with 32 bits (next block = block + grid stride).
-constexpr int64_t kMaxBlocksPerLaunch = 0x7FFF0000;
-
 bool block_size_ok(int B) { return B == 256 || B == 512 || B == 1024 || B == 2048 || B == 4096; }
 
-int log2_int(int v) {
-  int s = 0;
-  while ((1 << s) < v) ++s;
-  return s;
-}
-
-int grid_for(int64_t blocks, int groups_per_cta, int sm_count) {
-  const int64_t want = (blocks + groups_per_cta - 1) / groups_per_cta;
-  return static_cast<int>(want < sm_count ? want : sm_count);
-}
-
-// Values per thread and threads per CTA for each operation and block size.  A group (B / VPT
-// threads) is at least one warp, and the groups tile the CTA.
-template <int B, int VPT_WANTED, int THREADS_WANTED> struct GeometryOf {
-  static constexpr int VPT = (B / VPT_WANTED >= 32) ? VPT_WANTED : B / 32;
-  static constexpr int THREADS = (THREADS_WANTED % (B / VPT) == 0) ? THREADS_WANTED : (B / VPT);
-  static_assert(VPT % 4 == 0 && THREADS <= kCtaThreads && THREADS % (B / VPT) == 0, "bad geometry");
-};
-// The steps run 512 threads x 16 values.  Small blocks are latency-bound rather than issue-bound
-// (one warp owns a block): 768 threads with 8 values each measured 1-5 % faster there.
-template <int B> struct AdamGeometry : GeometryOf<B, 16, 512> {};
-template <> struct AdamGeometry<256> : GeometryOf<256, 8, 768> {};
-template <> struct AdamGeometry<512> : GeometryOf<512, 8, 768> {};
-template <int B> struct SgdGeometry : GeometryOf<B, 16, 512> {};
-template <> struct SgdGeometry<256> : GeometryOf<256, 8, 768> {};
-template <int B> using QuantGeometry = GeometryOf<B, 16, 1024>;
+bool dtype_ok(int d) { return d == DT8_F32 || d == DT8_BF16; }
 
 // Hyper-parameters are checked before anything is launched: non-finite values and decay rates
 // outside [0, 1) (1 - beta^step would be 0 or negative) are argument errors.
@@ -149,115 +148,16 @@ bool sgd_hyper_ok(float lr, float momentum, float wd) {
   return finite_all({lr, momentum, wd}) && momentum >= 0.0f;
 }
 
-int check_tensor(const TensorDesc& d, int g_dtype, bool adam) {
+int check_tensor(const TensorDesc& d, int p_dtype, int g_dtype, bool adam) {
   if (d.n < 0) return DT8_ERR_INVALID_ARG;
   if (d.n == 0) return DT8_OK;
   if (!d.p || !d.g || !d.mc || !d.ma) return DT8_ERR_INVALID_ARG;
   if (adam && (!d.rc || !d.ra)) return DT8_ERR_INVALID_ARG;
-  if (!aligned(d.p, 16) || !aligned(d.g, g_dtype == DT8_F32 ? 16 : 8) || !aligned(d.mc, 4) ||
-      !aligned(d.ma, 4))
+  if (!aligned(d.p, p_dtype == DT8_F32 ? 16 : 8) || !aligned(d.g, g_dtype == DT8_F32 ? 16 : 8) ||
+      !aligned(d.mc, 4) || !aligned(d.ma, 4))
     return DT8_ERR_ALIGNMENT;
   if (adam && (!aligned(d.rc, 4) || !aligned(d.ra, 4))) return DT8_ERR_ALIGNMENT;
   return DT8_OK;
-}
-
-// ---- launchers -------------------------------------------------------------------------------
-template <class Args, int B, bool GBF16, int MODE>
-int launch_adam(const Args& args, int64_t blocks, const AdamHyper& h, const EncMeta& em,
-                const DeviceInfo& di, cudaStream_t stream) {
-  constexpr int VPT = AdamGeometry<B>::VPT, THREADS = AdamGeometry<B>::THREADS;
-  constexpr int GROUPS = THREADS / (B / VPT);
-  auto kernel = block_kernel<AdamOp<B, VPT, THREADS, GBF16, MODE>, Args>;
-  const size_t smem = smem_bytes(em, true, true, true, true);
-  static std::atomic<uint64_t> smem_ok{0};
-  cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
-  if (e != cudaSuccess) return cuda_fail(e);
-  kernel<<<grid_for(blocks, GROUPS, di.sm_count), THREADS, smem, stream>>>(args, h, em);
-  e = cudaGetLastError();
-  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
-}
-
-template <class Args, int B, bool GBF16>
-int dispatch_adam_mode(const Args& args, int64_t blocks, int mode, const AdamHyper& h,
-                       const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
-  switch (mode) {
-    case kAdamWFast: return launch_adam<Args, B, GBF16, kAdamWFast>(args, blocks, h, em, di, s);
-    case kAdamWIeee: return launch_adam<Args, B, GBF16, kAdamWIeee>(args, blocks, h, em, di, s);
-    case kAdamWSmall: return launch_adam<Args, B, GBF16, kAdamWSmall>(args, blocks, h, em, di, s);
-    default: return launch_adam<Args, B, GBF16, kAdamL2>(args, blocks, h, em, di, s);
-  }
-}
-
-template <class Args, int B>
-int dispatch_adam(const Args& args, int64_t blocks, int g_dtype, int mode, const AdamHyper& h,
-                  const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
-  return g_dtype == DT8_BF16 ? dispatch_adam_mode<Args, B, true>(args, blocks, mode, h, em, di, s)
-                             : dispatch_adam_mode<Args, B, false>(args, blocks, mode, h, em, di, s);
-}
-
-template <class Args>
-int dispatch_adam_b(const Args& args, int64_t blocks, int B, int g_dtype, int mode,
-                    const AdamHyper& h, const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
-  switch (B) {
-    case 256: return dispatch_adam<Args, 256>(args, blocks, g_dtype, mode, h, em, di, s);
-    case 512: return dispatch_adam<Args, 512>(args, blocks, g_dtype, mode, h, em, di, s);
-    case 1024: return dispatch_adam<Args, 1024>(args, blocks, g_dtype, mode, h, em, di, s);
-    case 2048: return dispatch_adam<Args, 2048>(args, blocks, g_dtype, mode, h, em, di, s);
-    case 4096: return dispatch_adam<Args, 4096>(args, blocks, g_dtype, mode, h, em, di, s);
-  }
-  return DT8_ERR_UNSUPPORTED;
-}
-
-template <class Args, int B, bool GBF16>
-int launch_sgd(const Args& args, int64_t blocks, const SgdHyper& h, const EncMeta& em,
-               const DeviceInfo& di, cudaStream_t stream) {
-  constexpr int VPT = SgdGeometry<B>::VPT, THREADS = SgdGeometry<B>::THREADS;
-  constexpr int GROUPS = THREADS / (B / VPT);
-  auto kernel = block_kernel<SgdOp<B, VPT, THREADS, GBF16>, Args>;
-  const size_t smem = smem_bytes(em, true, false, true, true);
-  static std::atomic<uint64_t> smem_ok{0};
-  cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
-  if (e != cudaSuccess) return cuda_fail(e);
-  kernel<<<grid_for(blocks, GROUPS, di.sm_count), THREADS, smem, stream>>>(args, h, em);
-  e = cudaGetLastError();
-  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
-}
-
-template <class Args>
-int dispatch_sgd_b(const Args& args, int64_t blocks, int B, int g_dtype, const SgdHyper& h,
-                   const EncMeta& em, const DeviceInfo& di, cudaStream_t s) {
-#define DT8_SGD_CASE(BS)                                                        \
-  case BS:                                                                      \
-    return g_dtype == DT8_BF16 ? launch_sgd<Args, BS, true>(args, blocks, h, em, di, s) \
-                               : launch_sgd<Args, BS, false>(args, blocks, h, em, di, s);
-  switch (B) {
-    DT8_SGD_CASE(256)
-    DT8_SGD_CASE(512)
-    DT8_SGD_CASE(1024)
-    DT8_SGD_CASE(2048)
-    DT8_SGD_CASE(4096)
-  }
-#undef DT8_SGD_CASE
-  return DT8_ERR_UNSUPPORTED;
-}
-
-template <int B, bool SIGNED>
-int launch_quantize(const float* x, int64_t n, uint8_t* codes, float* absmax, const EncMeta& em,
-                    const DeviceInfo& di, cudaStream_t stream) {
-  constexpr int VPT = QuantGeometry<B>::VPT, THREADS = QuantGeometry<B>::THREADS;
-  constexpr int GROUPS = THREADS / (B / VPT);
-  auto kernel = block_kernel<QuantOp<B, VPT, THREADS, SIGNED>, SingleArgs>;
-  const size_t smem = smem_bytes(em, SIGNED, !SIGNED, false, true);
-  static std::atomic<uint64_t> smem_ok{0};
-  cudaError_t e = allow_smem(smem_ok, kernel, di.device, smem);
-  if (e != cudaSuccess) return cuda_fail(e);
-  SingleArgs a;
-  a.t = TensorDesc{nullptr, x, codes, absmax, nullptr, nullptr, n};
-  a.nb = (n + B - 1) / B;
-  if (a.nb > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
-  kernel<<<grid_for(a.nb, GROUPS, di.sm_count), THREADS, smem, stream>>>(a, NoHyper{0}, em);
-  e = cudaGetLastError();
-  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
 
 // Correctly rounded binary32 reciprocal of a positive normal binary32 number, on the host.  The
@@ -336,6 +236,27 @@ int adam_mode(uint32_t flags, const AdamHyper& h) {
 }
 
 }  // namespace
+
+template <class Args>
+static int launch_adam_any(const Args& a, int64_t blocks, int block_size, int p_dtype, int g_dtype,
+                           int mode, const AdamHyper& h, const LaunchCtx& ctx) {
+  const bool gb = g_dtype == DT8_BF16, pb = p_dtype == DT8_BF16;
+  if (gb && pb) return launch_adam_typed<true, true, Args>(a, blocks, block_size, mode, h, ctx);
+  if (gb) return launch_adam_typed<true, false, Args>(a, blocks, block_size, mode, h, ctx);
+  if (pb) return launch_adam_typed<false, true, Args>(a, blocks, block_size, mode, h, ctx);
+  return launch_adam_typed<false, false, Args>(a, blocks, block_size, mode, h, ctx);
+}
+
+int launch_adam(const SingleArgs& a, int64_t blocks, int block_size, int p_dtype, int g_dtype, int mode,
+                const AdamHyper& h, const LaunchCtx& ctx) {
+  return launch_adam_any(a, blocks, block_size, p_dtype, g_dtype, mode, h, ctx);
+}
+
+int launch_adam(const MultiArgs& a, int64_t blocks, int block_size, int p_dtype, int g_dtype, int mode,
+                const AdamHyper& h, const LaunchCtx& ctx) {
+  return launch_adam_any(a, blocks, block_size, p_dtype, g_dtype, mode, h, ctx);
+}
+
 }  // namespace dt8
 
 using namespace dt8;
@@ -396,10 +317,10 @@ int dt8_selfcheck_encode_host(int is_signed, const float* v_host, int64_t n, uin
   return DT8_OK;
 }
 
+
 int dt8_init(void) {
-  DeviceInfo di;
-  EncMeta em;
-  return ensure_device(&di, &em);
+  LaunchCtx ctx;
+  return ensure_device(&ctx, nullptr);
 }
 
 int dt8_selfcheck_divide(const float* s, const float* N, int64_t n, float* out, void* stream) {
@@ -407,13 +328,12 @@ int dt8_selfcheck_divide(const float* s, const float* N, int64_t n, float* out, 
   if (n == 0) return DT8_OK;
   if (!s || !N || !out) return DT8_ERR_INVALID_ARG;
   if (!aligned(s, 4) || !aligned(N, 4) || !aligned(out, 4)) return DT8_ERR_ALIGNMENT;
-  DeviceInfo di;
-  EncMeta em;
-  int rc = ensure_device(&di, &em);
+  LaunchCtx ctx;
+  int rc = ensure_device(&ctx, stream);
   if (rc != DT8_OK) return rc;
   const int64_t ctas = (n + 255) / 256;
-  const int grid = static_cast<int>(ctas < 8 * di.sm_count ? ctas : 8 * di.sm_count);
-  divide_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(s, N, out, n);
+  const int grid = static_cast<int>(ctas < 8 * ctx.sm_count ? ctas : 8 * ctx.sm_count);
+  divide_kernel<<<grid, 256, 0, ctx.stream>>>(s, N, out, n);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
@@ -423,13 +343,12 @@ int dt8_selfcheck_divide_const(const float* s, float d, int64_t n, float* out, v
   if (n == 0) return DT8_OK;
   if (!s || !out) return DT8_ERR_INVALID_ARG;
   if (!aligned(s, 4) || !aligned(out, 4)) return DT8_ERR_ALIGNMENT;
-  DeviceInfo di;
-  EncMeta em;
-  int rc = ensure_device(&di, &em);
+  LaunchCtx ctx;
+  int rc = ensure_device(&ctx, stream);
   if (rc != DT8_OK) return rc;
   const int64_t ctas = (n + 255) / 256;
-  const int grid = static_cast<int>(ctas < 8 * di.sm_count ? ctas : 8 * di.sm_count);
-  divide_const_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(s, make_const_divisor(d), out, n);
+  const int grid = static_cast<int>(ctas < 8 * ctx.sm_count ? ctas : 8 * ctx.sm_count);
+  divide_const_kernel<<<grid, 256, 0, ctx.stream>>>(s, make_const_divisor(d), out, n);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }
@@ -441,24 +360,11 @@ int dt8_quantize_blockwise(const float* x, int64_t n, int block_size, int is_sig
   if (n == 0) return DT8_OK;
   if (!x || !codes || !absmax) return DT8_ERR_INVALID_ARG;
   if (!aligned(x, 16) || !aligned(codes, 4) || !aligned(absmax, 4)) return DT8_ERR_ALIGNMENT;
-  DeviceInfo di;
-  EncMeta em;
-  int rc = ensure_device(&di, &em);
+  if ((n + block_size - 1) / block_size > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
+  LaunchCtx ctx;
+  int rc = ensure_device(&ctx, stream);
   if (rc != DT8_OK) return rc;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define DT8_Q_CASE(BS)                                                                  \
-  case BS:                                                                              \
-    return is_signed ? launch_quantize<BS, true>(x, n, codes, absmax, em, di, s)        \
-                     : launch_quantize<BS, false>(x, n, codes, absmax, em, di, s);
-  switch (block_size) {
-    DT8_Q_CASE(256)
-    DT8_Q_CASE(512)
-    DT8_Q_CASE(1024)
-    DT8_Q_CASE(2048)
-    DT8_Q_CASE(4096)
-  }
-#undef DT8_Q_CASE
-  return DT8_ERR_UNSUPPORTED;
+  return launch_quantize(x, n, block_size, is_signed, codes, absmax, ctx);
 }
 
 int dt8_dequantize_blockwise(const uint8_t* codes, const float* absmax, int64_t n, int block_size,
@@ -468,66 +374,65 @@ int dt8_dequantize_blockwise(const uint8_t* codes, const float* absmax, int64_t 
   if (n == 0) return DT8_OK;
   if (!codes || !absmax || !out) return DT8_ERR_INVALID_ARG;
   if (!aligned(out, 16) || !aligned(codes, 4) || !aligned(absmax, 4)) return DT8_ERR_ALIGNMENT;
-  DeviceInfo di;
-  EncMeta em;
-  int rc = ensure_device(&di, &em);
+  LaunchCtx ctx;
+  int rc = ensure_device(&ctx, stream);
   if (rc != DT8_OK) return rc;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int64_t quads = (n + 3) / 4;
-  const int64_t per_cta = static_cast<int64_t>(kDeqThreads) * kDeqUnroll;
-  const int64_t ctas = (quads + per_cta - 1) / per_cta;
-  const int64_t resident = static_cast<int64_t>(kDeqCtasPerSm) * di.sm_count;
-  const int grid = static_cast<int>(ctas < resident ? ctas : resident);
-  const int shift = log2_int(block_size);
-  if (is_signed)
-    dequantize_kernel<true><<<grid, kDeqThreads, kDeqSmemBytes, s>>>(codes, absmax, out, n, shift);
-  else
-    dequantize_kernel<false><<<grid, kDeqThreads, kDeqSmemBytes, s>>>(codes, absmax, out, n, shift);
-  const cudaError_t e = cudaGetLastError();
-  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+  return launch_dequantize(codes, absmax, n, block_size, is_signed, out, ctx);
+}
+
+int dt8_sgd_step_ex(void* p, int p_dtype, const void* g, int g_dtype, uint8_t* m_codes,
+                    float* m_absmax, int64_t n, float lr, float momentum, float weight_decay,
+                    int64_t step, int block_size, void* stream) {
+  if (!dtype_ok(g_dtype) || !dtype_ok(p_dtype)) return DT8_ERR_INVALID_ARG;
+  if (step < 1 || !sgd_hyper_ok(lr, momentum, weight_decay)) return DT8_ERR_INVALID_ARG;
+  if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
+  SingleArgs a;
+  a.t = TensorDesc{p, g, m_codes, m_absmax, nullptr, nullptr, n};
+  int rc = check_tensor(a.t, p_dtype, g_dtype, false);
+  if (rc != DT8_OK || n == 0) return rc;
+  a.nb = (n + block_size - 1) / block_size;
+  if (a.nb > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
+  LaunchCtx ctx;
+  rc = ensure_device(&ctx, stream);
+  if (rc != DT8_OK) return rc;
+  const SgdHyper h{lr, momentum, weight_decay};
+  return launch_sgd(a, a.nb, block_size, p_dtype, g_dtype, h, ctx);
 }
 
 int dt8_sgd_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float* m_absmax, int64_t n,
                  float lr, float momentum, float weight_decay, int64_t step, int block_size,
                  void* stream) {
-  if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
-  if (step < 1 || !sgd_hyper_ok(lr, momentum, weight_decay)) return DT8_ERR_INVALID_ARG;
+  return dt8_sgd_step_ex(p, DT8_F32, g, g_dtype, m_codes, m_absmax, n, lr, momentum, weight_decay,
+                         step, block_size, stream);
+}
+
+int dt8_adam_step_ex(void* p, int p_dtype, const void* g, int g_dtype, uint8_t* m_codes,
+                     float* m_absmax, uint8_t* r_codes, float* r_absmax, int64_t n, float lr,
+                     float beta1, float beta2, float eps, float weight_decay, int64_t step,
+                     int block_size, uint32_t flags, void* stream) {
+  if (!dtype_ok(g_dtype) || !dtype_ok(p_dtype)) return DT8_ERR_INVALID_ARG;
+  if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
+  if (!adam_hyper_ok(lr, beta1, beta2, eps, weight_decay)) return DT8_ERR_INVALID_ARG;
   if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
   SingleArgs a;
-  a.t = TensorDesc{p, g, m_codes, m_absmax, nullptr, nullptr, n};
-  int rc = check_tensor(a.t, g_dtype, false);
+  a.t = TensorDesc{p, g, m_codes, m_absmax, r_codes, r_absmax, n};
+  int rc = check_tensor(a.t, p_dtype, g_dtype, true);
   if (rc != DT8_OK || n == 0) return rc;
   a.nb = (n + block_size - 1) / block_size;
   if (a.nb > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
-  DeviceInfo di;
-  EncMeta em;
-  rc = ensure_device(&di, &em);
+  LaunchCtx ctx;
+  rc = ensure_device(&ctx, stream);
   if (rc != DT8_OK) return rc;
-  const SgdHyper h{lr, momentum, weight_decay};
-  return dispatch_sgd_b(a, a.nb, block_size, g_dtype, h, em, di, static_cast<cudaStream_t>(stream));
+  const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
+  return launch_adam(a, a.nb, block_size, p_dtype, g_dtype, adam_mode(flags, h), h, ctx);
 }
 
 int dt8_adam_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float* m_absmax,
                   uint8_t* r_codes, float* r_absmax, int64_t n, float lr, float beta1, float beta2,
                   float eps, float weight_decay, int64_t step, int block_size, uint32_t flags,
                   void* stream) {
-  if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
-  if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
-  if (!adam_hyper_ok(lr, beta1, beta2, eps, weight_decay)) return DT8_ERR_INVALID_ARG;
-  if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
-  SingleArgs a;
-  a.t = TensorDesc{p, g, m_codes, m_absmax, r_codes, r_absmax, n};
-  int rc = check_tensor(a.t, g_dtype, true);
-  if (rc != DT8_OK || n == 0) return rc;
-  a.nb = (n + block_size - 1) / block_size;
-  if (a.nb > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
-  DeviceInfo di;
-  EncMeta em;
-  rc = ensure_device(&di, &em);
-  if (rc != DT8_OK) return rc;
-  const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
-  return dispatch_adam_b(a, a.nb, block_size, g_dtype, adam_mode(flags, h), h, em, di,
-                         static_cast<cudaStream_t>(stream));
+  return dt8_adam_step_ex(p, DT8_F32, g, g_dtype, m_codes, m_absmax, r_codes, r_absmax, n, lr, beta1,
+                          beta2, eps, weight_decay, step, block_size, flags, stream);
 }
 
 }  // extern "C"
@@ -535,29 +440,28 @@ int dt8_adam_step(float* p, const void* g, int g_dtype, uint8_t* m_codes, float*
 namespace dt8 {
 namespace {
 
-// Shared front end of the two pointer-list entry points: validates every tensor first (so that a
+// Shared front end of the pointer-list entry points: validates every tensor first (so that a
 // bad entry means nothing was launched), then launches one kernel per kMaxTensorsPerLaunch
 // non-empty tensors.  Every tensor that passed the checks fits a launch of its own, so after the
 // checks only the CUDA runtime can fail (DT8_ERR_CUDA), possibly after earlier launches of the
 // same call were queued.
 template <class Launch>
-int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtype,
+int run_multi(int num_tensors, void* const* p, int p_dtype, const void* const* g, int g_dtype,
               uint8_t* const* mc, float* const* ma, uint8_t* const* rc, float* const* ra,
-              const int64_t* n, int block_size, bool adam, Launch launch) {
+              const int64_t* n, int block_size, bool adam, void* stream, Launch launch) {
   if (num_tensors < 0) return DT8_ERR_INVALID_ARG;
-  if (g_dtype != DT8_F32 && g_dtype != DT8_BF16) return DT8_ERR_INVALID_ARG;
+  if (!dtype_ok(g_dtype) || !dtype_ok(p_dtype)) return DT8_ERR_INVALID_ARG;
   if (!block_size_ok(block_size)) return DT8_ERR_UNSUPPORTED;
   if (num_tensors == 0) return DT8_OK;
   if (!p || !g || !mc || !ma || !n || (adam && (!rc || !ra))) return DT8_ERR_INVALID_ARG;
   for (int i = 0; i < num_tensors; ++i) {
     const TensorDesc d{p[i], g[i], mc[i], ma[i], adam ? rc[i] : nullptr, adam ? ra[i] : nullptr, n[i]};
-    const int st = check_tensor(d, g_dtype, adam);
+    const int st = check_tensor(d, p_dtype, g_dtype, adam);
     if (st != DT8_OK) return st;
     if ((n[i] + block_size - 1) / block_size > kMaxBlocksPerLaunch) return DT8_ERR_UNSUPPORTED;
   }
-  DeviceInfo di;
-  EncMeta em;
-  int st = ensure_device(&di, &em);
+  LaunchCtx ctx;
+  int st = ensure_device(&ctx, stream);
   if (st != DT8_OK) return st;
   static thread_local MultiArgs args;
   int i = 0;
@@ -577,7 +481,7 @@ int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtyp
       ++i;
     }
     if (args.num == 0) continue;
-    st = launch(args, blocks, em, di);
+    st = launch(args, blocks, ctx);
     if (st != DT8_OK) return st;
   }
   return DT8_OK;
@@ -588,16 +492,41 @@ int run_multi(int num_tensors, float* const* p, const void* const* g, int g_dtyp
 
 extern "C" {
 
+int dt8_sgd_step_multi_ex(int num_tensors, void* const* p, int p_dtype, const void* const* g,
+                          int g_dtype, uint8_t* const* m_codes, float* const* m_absmax,
+                          const int64_t* n, float lr, float momentum, float weight_decay,
+                          int64_t step, int block_size, void* stream) {
+  if (step < 1 || !sgd_hyper_ok(lr, momentum, weight_decay)) return DT8_ERR_INVALID_ARG;
+  const SgdHyper h{lr, momentum, weight_decay};
+  return run_multi(num_tensors, p, p_dtype, g, g_dtype, m_codes, m_absmax, nullptr, nullptr, n,
+                   block_size, false, stream,
+                   [&](const MultiArgs& a, int64_t blocks, const LaunchCtx& ctx) {
+                     return launch_sgd(a, blocks, block_size, p_dtype, g_dtype, h, ctx);
+                   });
+}
+
 int dt8_sgd_step_multi(int num_tensors, float* const* p, const void* const* g, int g_dtype,
                        uint8_t* const* m_codes, float* const* m_absmax, const int64_t* n, float lr,
                        float momentum, float weight_decay, int64_t step, int block_size,
                        void* stream) {
-  if (step < 1 || !sgd_hyper_ok(lr, momentum, weight_decay)) return DT8_ERR_INVALID_ARG;
-  const SgdHyper h{lr, momentum, weight_decay};
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  return run_multi(num_tensors, p, g, g_dtype, m_codes, m_absmax, nullptr, nullptr, n, block_size,
-                   false, [&](const MultiArgs& a, int64_t blocks, const EncMeta& em, const DeviceInfo& di) {
-                     return dispatch_sgd_b(a, blocks, block_size, g_dtype, h, em, di, s);
+  return dt8_sgd_step_multi_ex(num_tensors, reinterpret_cast<void* const*>(p), DT8_F32, g, g_dtype,
+                               m_codes, m_absmax, n, lr, momentum, weight_decay, step, block_size,
+                               stream);
+}
+
+int dt8_adam_step_multi_ex(int num_tensors, void* const* p, int p_dtype, const void* const* g,
+                           int g_dtype, uint8_t* const* m_codes, float* const* m_absmax,
+                           uint8_t* const* r_codes, float* const* r_absmax, const int64_t* n,
+                           float lr, float beta1, float beta2, float eps, float weight_decay,
+                           int64_t step, int block_size, uint32_t flags, void* stream) {
+  if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
+  if (!adam_hyper_ok(lr, beta1, beta2, eps, weight_decay)) return DT8_ERR_INVALID_ARG;
+  const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
+  const int mode = adam_mode(flags, h);
+  return run_multi(num_tensors, p, p_dtype, g, g_dtype, m_codes, m_absmax, r_codes, r_absmax, n,
+                   block_size, true, stream,
+                   [&](const MultiArgs& a, int64_t blocks, const LaunchCtx& ctx) {
+                     return launch_adam(a, blocks, block_size, p_dtype, g_dtype, mode, h, ctx);
                    });
 }
 
@@ -606,15 +535,9 @@ int dt8_adam_step_multi(int num_tensors, float* const* p, const void* const* g, 
                         float* const* r_absmax, const int64_t* n, float lr, float beta1, float beta2,
                         float eps, float weight_decay, int64_t step, int block_size, uint32_t flags,
                         void* stream) {
-  if (step < 1 || (flags & ~3u)) return DT8_ERR_INVALID_ARG;
-  if (!adam_hyper_ok(lr, beta1, beta2, eps, weight_decay)) return DT8_ERR_INVALID_ARG;
-  const AdamHyper h = make_adam_hyper(lr, beta1, beta2, eps, weight_decay, step, flags);
-  const int mode = adam_mode(flags, h);
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  return run_multi(num_tensors, p, g, g_dtype, m_codes, m_absmax, r_codes, r_absmax, n, block_size,
-                   true, [&](const MultiArgs& a, int64_t blocks, const EncMeta& em, const DeviceInfo& di) {
-                     return dispatch_adam_b(a, blocks, block_size, g_dtype, mode, h, em, di, s);
-                   });
+  return dt8_adam_step_multi_ex(num_tensors, reinterpret_cast<void* const*>(p), DT8_F32, g, g_dtype,
+                                m_codes, m_absmax, r_codes, r_absmax, n, lr, beta1, beta2, eps,
+                                weight_decay, step, block_size, flags, stream);
 }
 
 }  // extern "C"

@@ -174,7 +174,7 @@ class _Scale(torch.nn.Module):
 def test_block_gradients_closed_form_for_scalar_branches():
     """With F(v) = a v and G(v) = b v, Eq. revnet4 gives y1 = x1 + a x2, y2 = x2 + b y1, hence
     dL/dx1 = dy1 + b dy2, dL/dx2 = a (dy1 + b dy2) + dy2, dL/da = sum((dy1 + b dy2) x2),
-    dL/db = sum(dy2 y1): the quantities lines 4-8 of Alg. 1 compute."""
+    dL/db = sum(dy2 y1): the quantities Alg. 1 returns."""
     a, b = 0.75, -1.5
     g = torch.Generator().manual_seed(5)
     x = torch.randn(2, 4, 3, 5, generator=g, dtype=torch.float64)
