@@ -22,9 +22,12 @@ def lib():
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "dt8.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(dt8_[a-z0-9_]+)\s*\(", text)))
+    import glob
+    names = set()
+    for path in glob.glob(os.path.join(ROOT, "include", "*.h")):
+        text = re.sub(r"/\*.*?\*/", "", open(path).read(), flags=re.S)
+        names |= set(re.findall(r"\b(dt8_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol(lib):
@@ -33,7 +36,9 @@ def test_library_exports_every_declared_symbol(lib):
             "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi"} <= set(names)
     for name in names:
         assert hasattr(lib, name), name
-    assert set(names) == set(dt8.EXPORTS)
+    from paper_2412_01195_b200 import rev
+    assert set(names) == set(dt8.EXPORTS) | set(rev.REV_EXPORTS)
+    assert set(rev.REV_EXPORTS) == {n for n in names if n.startswith("dt8_rev_")}
 
 
 def test_status_strings(lib):
@@ -207,6 +212,32 @@ def test_hyper_parameters_are_validated_before_any_device_work(lib):
                                   f(0), 1, 256, None) == E.DT8_ERR_UNSUPPORTED
     assert lib.dt8_sgd_step(ok, ok, 0, ok, ok, (0x7FFF0000 + 1) * 256, f(.1), f(.9), f(0), 1, 256,
                             None) == E.DT8_ERR_UNSUPPORTED
+
+
+def test_reversible_kernel_argument_checks_return_before_any_device_work(lib):
+    from paper_2412_01195_b200 import rev
+    rev._lib()
+    buf = (ctypes.c_uint8 * 4096)()
+    base = ctypes.addressof(buf)
+    ok, odd = ctypes.c_void_p(base + (-base) % 16), ctypes.c_void_p(base + (-base) % 16 + 2)
+    E = dt8
+    for fn in (lib.dt8_rev_coupling_forward, lib.dt8_rev_coupling_inverse):
+        assert fn(ok, ok, ok, -1, 8, 0, None) == E.DT8_ERR_INVALID_ARG
+        assert fn(ok, ok, ok, 2, -8, 0, None) == E.DT8_ERR_INVALID_ARG
+        assert fn(ok, ok, ok, 2, 8, 2, None) == E.DT8_ERR_INVALID_ARG
+        assert fn(None, ok, ok, 2, 8, 0, None) == E.DT8_ERR_INVALID_ARG
+        assert fn(odd, ok, ok, 2, 8, 0, None) == E.DT8_ERR_ALIGNMENT
+        assert fn(None, None, None, 0, 8, 0, None) == E.DT8_OK
+    s2d, d2s = lib.dt8_rev_space_to_depth, lib.dt8_rev_depth_to_space
+    assert s2d(ok, 1, 1, 3, 4, ok, None) == E.DT8_ERR_INVALID_ARG          # odd F
+    assert s2d(ok, 1, 1, 4, 5, ok, None) == E.DT8_ERR_INVALID_ARG          # odd T
+    assert s2d(ok, -1, 1, 4, 4, ok, None) == E.DT8_ERR_INVALID_ARG
+    assert s2d(None, 1, 1, 4, 4, ok, None) == E.DT8_ERR_INVALID_ARG
+    assert s2d(odd, 1, 1, 4, 4, ok, None) == E.DT8_ERR_ALIGNMENT
+    assert s2d(ok, 1 << 20, 1 << 10, 4, 4, ok, None) == E.DT8_ERR_UNSUPPORTED   # 2^34 elements
+    assert s2d(None, 0, 4, 4, 4, None, None) == E.DT8_OK
+    assert d2s(ok, 1, 1, -2, 2, ok, None) == E.DT8_ERR_INVALID_ARG
+    assert d2s(None, 1, 4, 0, 2, None, None) == E.DT8_OK
 
 
 class _NoLaunch:
