@@ -1,19 +1,22 @@
 """Block-range-sharded 8-bit Adam step for data-parallel training.
 
-Quantization blocks are independent (Section IV-B: "quantization applied independently to each
-block") and the update is element-wise, so the optimizer state of a flat parameter buffer can be
-split across the ranks of a data-parallel job on block boundaries with no exchange inside the
-step.  Around the step sit the two collectives every sharded optimizer needs:
+Every quantization block is quantized on its own (Section IV-B, "Tensor chunking") and the update
+is element-wise, so the optimizer state of a flat parameter buffer can be split across the ranks
+of a data-parallel job on block boundaries with no exchange inside the step.  Around the step sit
+the two collectives every sharded optimizer needs:
 
     reduce-scatter(gradients)  ->  dt8_adam_step on the owned block range  ->  all-gather(parameters)
 
 `torch.distributed` supplies the collectives (NCCL on GPUs); the step itself is the CUDA library.
 Each rank keeps the 8-bit states of its own range only: state memory per rank is
 (n + 4n/B) * 2 / world_size bytes for Adam.
+
+Which collectives are issued is decided once, from the backend of the process group: NCCL has
+reduce-scatter with averaging and all-gather into one tensor; gloo has neither, so there the
+gradients are all-reduced and the parameters gathered as a list.  Errors of a collective are
+never caught: a rank that took another path than its peers would leave them waiting.
 """
 from __future__ import annotations
-
-from typing import Callable, Optional
 
 import torch
 import torch.distributed as dist
@@ -39,14 +42,16 @@ class ShardedAdam8bit:
     `params` holds the padded parameters (length `padded`), `grads` the local gradients of the
     same length; `step()` averages the gradients over the ranks into this rank's shard, steps the
     shard in place and gathers the updated parameters back into `params` on every rank.
-    `step_fn` and `state_fn` exist so that the plumbing can be exercised without a GPU.
     """
 
-    def __init__(self, n: int, block_size: int = 2048, device="cuda", group=None,
-                 step_fn: Optional[Callable] = None, state_fn: Optional[Callable] = None):
+    def __init__(self, n: int, block_size: int = 2048, device="cuda", group=None):
         self.group = group
-        self.rank = dist.get_rank(group) if dist.is_initialized() else 0
-        self.world = dist.get_world_size(group) if dist.is_initialized() else 1
+        ready = dist.is_available() and dist.is_initialized()
+        self.rank = dist.get_rank(group) if ready else 0
+        self.world = dist.get_world_size(group) if ready else 1
+        self.backend = dist.get_backend(group) if ready else "none"
+        # tensor collectives (reduce_scatter_tensor with AVG, all_gather_into_tensor) are NCCL's
+        self.tensor_collectives = self.backend == "nccl"
         self.n, self.block_size = n, block_size
         self.blocks, self.per_rank, self.padded = shard_layout(n, block_size, self.world)
         self.params = torch.zeros(self.padded, dtype=torch.float32, device=device)
@@ -54,41 +59,44 @@ class ShardedAdam8bit:
         self._gshard = torch.empty(self.per_rank, dtype=torch.float32, device=device)
         lo = self.rank * self.per_rank
         self.shard = self.params[lo:lo + self.per_rank]          # a view: stepped in place
-        make = state_fn or dt8.new_state
-        self.m_codes, self.m_absmax = make(self.per_rank, block_size, True, device)
-        self.r_codes, self.r_absmax = make(self.per_rank, block_size, False, device)
-        self._step_fn = step_fn or dt8.dt8_adam_step
+        self.m_codes, self.m_absmax = self._new_state(True, device)
+        self.r_codes, self.r_absmax = self._new_state(False, device)
         self.steps = 0
+
+    def _new_state(self, signed: bool, device):
+        return dt8.new_state(self.per_rank, self.block_size, signed, device)
+
+    def _step_shard(self, lr, beta1, beta2, eps, weight_decay, flags) -> None:
+        dt8.dt8_adam_step(self.shard, self._gshard, self.m_codes, self.m_absmax, self.r_codes,
+                          self.r_absmax, lr, beta1, beta2, eps, weight_decay, self.steps,
+                          self.block_size, flags)
 
     def state_bytes(self) -> int:
         """Bytes of optimizer state held by this rank."""
         return 2 * dt8.dt8_state_bytes(self.per_rank, self.block_size)
 
-    def _reduce_scatter_mean(self):
+    def _reduce_scatter_mean(self) -> None:
         if self.world == 1:
             self._gshard.copy_(self.grads)
-            return
-        try:
-            dist.reduce_scatter_tensor(self._gshard, self.grads, op=dist.ReduceOp.SUM, group=self.group)
-        except (RuntimeError, NotImplementedError):
-            # backends without reduce-scatter (gloo on CPU): all-reduce, then keep the own range
-            total = self.grads.clone()
-            dist.all_reduce(total, op=dist.ReduceOp.SUM, group=self.group)
+        elif self.tensor_collectives:
+            dist.reduce_scatter_tensor(self._gshard, self.grads, op=dist.ReduceOp.AVG, group=self.group)
+        else:
+            dist.all_reduce(self.grads, op=dist.ReduceOp.SUM, group=self.group)
             lo = self.rank * self.per_rank
-            self._gshard.copy_(total[lo:lo + self.per_rank])
-        self._gshard.div_(self.world)
+            torch.div(self.grads[lo:lo + self.per_rank], self.world, out=self._gshard)
+
+    def _all_gather_params(self) -> None:
+        if self.world == 1:
+            return
+        if self.tensor_collectives:
+            # in place: this rank's shard already sits at its position of the output
+            dist.all_gather_into_tensor(self.params, self.shard, group=self.group)
+        else:
+            parts = list(self.params.split(self.per_rank))
+            dist.all_gather(parts, self.shard.clone(), group=self.group)
 
     def step(self, lr, beta1, beta2, eps, weight_decay, flags=dt8.DEFAULT_ADAM_FLAGS) -> None:
         self.steps += 1
         self._reduce_scatter_mean()
-        self._step_fn(self.shard, self._gshard, self.m_codes, self.m_absmax, self.r_codes,
-                      self.r_absmax, lr, beta1, beta2, eps, weight_decay, self.steps,
-                      self.block_size, flags)
-        if self.world > 1:
-            mine = self.shard.clone()
-            try:
-                dist.all_gather_into_tensor(self.params, mine, group=self.group)
-            except (RuntimeError, NotImplementedError):
-                parts = [torch.empty_like(mine) for _ in range(self.world)]
-                dist.all_gather(parts, mine, group=self.group)
-                self.params.copy_(torch.cat(parts))
+        self._step_shard(lr, beta1, beta2, eps, weight_decay, flags)
+        self._all_gather_params()
