@@ -50,12 +50,34 @@ int launch_quantize(const float* x, int64_t n, int block_size, int is_signed, ui
 
 int launch_dequantize(const uint8_t* codes, const float* absmax, int64_t n, int block_size,
                       int is_signed, float* out, const LaunchCtx& ctx) {
+  // whole tiles: the bulk-store kernel; what is left (less than one tile): per-thread stores
+  const int shift = log2_int(block_size);
+  const int64_t tiles = n / kDeqBulkTile;
+  if (tiles > 0) {
+    static std::atomic<uint64_t> ok_s{0}, ok_u{0};
+    cudaError_t e = is_signed ? allow_smem(ok_s, dequantize_bulk_kernel<true>, ctx.device, kDeqBulkSmemBytes)
+                              : allow_smem(ok_u, dequantize_bulk_kernel<false>, ctx.device, kDeqBulkSmemBytes);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const int64_t resident = static_cast<int64_t>(kDeqBulkCtasPerSm) * ctx.sm_count;
+    const int g = static_cast<int>(tiles < resident ? tiles : resident);
+    if (is_signed)
+      dequantize_bulk_kernel<true><<<g, kDeqBulkThreads, kDeqBulkSmemBytes, ctx.stream>>>(codes, absmax, out, tiles, shift, ctx.tables);
+    else
+      dequantize_bulk_kernel<false><<<g, kDeqBulkThreads, kDeqBulkSmemBytes, ctx.stream>>>(codes, absmax, out, tiles, shift, ctx.tables);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    const int64_t done = tiles * kDeqBulkTile;     // a multiple of every block size
+    codes += done;
+    out += done;
+    absmax += done >> shift;
+    n -= done;
+    if (n == 0) return DT8_OK;
+  }
   const int64_t quads = (n + 3) / 4;
   const int64_t per_cta = static_cast<int64_t>(kDeqThreads) * kDeqUnroll;
   const int64_t ctas = (quads + per_cta - 1) / per_cta;
   const int64_t resident = static_cast<int64_t>(kDeqCtasPerSm) * ctx.sm_count;
   const int grid = static_cast<int>(ctas < resident ? ctas : resident);
-  const int shift = log2_int(block_size);
   if (is_signed)
     dequantize_kernel<true><<<grid, kDeqThreads, kDeqSmemBytes, ctx.stream>>>(codes, absmax, out, n, shift, ctx.tables);
   else
