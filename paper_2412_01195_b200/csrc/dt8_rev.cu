@@ -199,6 +199,85 @@ shuffle_kernel(const float* __restrict__ src, float* __restrict__ dst, uint32_t 
   }
 }
 
+// Rows that are not a multiple of 4 floats (T = 50 in the paper's last down-sampling stage) leave
+// the output rows at 4-byte alignment only.  A channel plane, however, occupies the same
+// contiguous range on both sides (F * T floats, a multiple of 4), so small planes are permuted in
+// shared memory: a CTA copies a run of whole planes in with 16-byte loads, and writes the same
+// range out with 16-byte stores, each output element gathered from its source position.
+constexpr int kPlaneThreads = 256;
+constexpr int kPlaneTileFloats = 6144;    // 24 KB of dynamic shared memory: eight CTAs per SM
+
+struct PlaneMap {
+  FastDiv plane;   // F * T
+  FastDiv chan;    // Fo * To
+  FastDiv row;     // To (to depth) or T (from depth)
+  uint32_t F, T;
+};
+
+template <bool TO_DEPTH>
+__global__ void __launch_bounds__(kPlaneThreads)
+shuffle_planes_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t planes,
+                      int planes_per_tile, PlaneMap m) {
+  extern __shared__ __align__(16) float plane_buf[];
+  const uint32_t PS = m.plane.d, To = m.T >> 1, Fo = m.F >> 1;
+  const int64_t tiles = (planes + planes_per_tile - 1) / planes_per_tile;
+  for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const int64_t first = tile * planes_per_tile;
+    const int64_t left = planes - first;
+    const uint32_t count = static_cast<uint32_t>(left < planes_per_tile ? left : planes_per_tile) * PS;
+    const float4* in4 = reinterpret_cast<const float4*>(src + first * PS);
+    float4* out4 = reinterpret_cast<float4*>(dst + first * PS);
+    // four independent loads in flight per thread
+    for (uint32_t i0 = threadIdx.x; i0 < count / 4; i0 += 4 * kPlaneThreads) {
+      float4 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (i0 + k * kPlaneThreads < count / 4) v[k] = __ldcs(in4 + i0 + k * kPlaneThreads);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (i0 + k * kPlaneThreads < count / 4) reinterpret_cast<float4*>(plane_buf)[i0 + k * kPlaneThreads] = v[k];
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < count / 4; i += kPlaneThreads) {
+      const uint32_t e = 4 * i;
+      const uint32_t p = m.plane.div(e);
+      uint32_t r = e - p * PS;
+      const float* base = plane_buf + p * PS;
+      float v[4];
+      if (TO_DEPTH) {
+        // output position (q, fo, to) of the plane <- input position (2 fo + q / 2, 2 to + q % 2)
+        uint32_t q = m.chan.div(r);
+        r -= q * m.chan.d;
+        uint32_t fo = m.row.div(r), to = r - fo * To;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          v[k] = base[(2 * fo + (q >> 1)) * m.T + 2 * to + (q & 1)];
+          if (++to == To) {
+            to = 0;
+            if (++fo == Fo) {
+              fo = 0;
+              ++q;
+            }
+          }
+        }
+      } else {
+        // output position (f, t) of the plane <- rearranged position (2 (f % 2) + t % 2, f / 2, t / 2)
+        uint32_t f = m.row.div(r), t = r - f * m.T;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          v[k] = base[((2 * (f & 1) + (t & 1)) * Fo + (f >> 1)) * To + (t >> 1)];
+          if (++t == m.T) {
+            t = 0;
+            ++f;
+          }
+        }
+      }
+      __stcs(out4 + i, make_float4(v[0], v[1], v[2], v[3]));
+    }
+    __syncthreads();
+  }
+}
+
 // `flat` is the N x C x F x T side, `deep` the N x 4C x F/2 x T/2 side.
 template <bool TO_DEPTH>
 int launch_shuffle(const float* src, float* dst, int64_t N, int64_t C, int64_t F, int64_t T, void* stream) {
@@ -222,13 +301,30 @@ int launch_shuffle(const float* src, float* dst, int64_t N, int64_t C, int64_t F
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return cuda_fail(e);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t plane = F * T;
+  if (!vec4 && plane <= kPlaneTileFloats && aligned_to(src, 16) && aligned_to(dst, 16)) {
+    // short rows, small planes: permute whole planes in shared memory
+    const int per_tile = static_cast<int>(kPlaneTileFloats / plane);
+    const uint32_t To = static_cast<uint32_t>(T / 2), Fo = static_cast<uint32_t>(F / 2);
+    PlaneMap pm{FastDiv(static_cast<uint32_t>(plane)), FastDiv(Fo * To),
+                FastDiv(TO_DEPTH ? To : static_cast<uint32_t>(T)), static_cast<uint32_t>(F),
+                static_cast<uint32_t>(T)};
+    const int64_t planes = N * C;
+    const int64_t tiles = (planes + per_tile - 1) / per_tile;
+    const int64_t cap = static_cast<int64_t>(sms) * 8;
+    const unsigned g = static_cast<unsigned>(tiles < cap ? tiles : cap);
+    const size_t smem = static_cast<size_t>(per_tile) * plane * sizeof(float);
+    shuffle_planes_kernel<TO_DEPTH><<<g, kPlaneThreads, smem, s>>>(src, dst, planes, per_tile, pm);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+  }
   ShuffleMap map{FastDiv(static_cast<uint32_t>(T / vec)), FastDiv(static_cast<uint32_t>(F)),
                  static_cast<uint32_t>(T), static_cast<uint32_t>(F)};
   const int64_t tile = static_cast<int64_t>(kShuffleThreads) * kShuffleUnroll;
   const int64_t want = (pieces + tile - 1) / tile;
   const int64_t cap = static_cast<int64_t>(sms) * 16;
   const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (vec4)
     shuffle_kernel<4, TO_DEPTH><<<grid, kShuffleThreads, 0, s>>>(src, dst, static_cast<uint32_t>(pieces), map);
   else
