@@ -392,6 +392,9 @@ def sub_cases():
     act = (128, 48, 80, 200)
     c = {
         "adam26": (lambda d: case_adam(d, 1 << 26), 50, "Adam, fp32 grads, 2^26 elements"),
+        "adam26_bf16grad": (lambda d: case_adam(d, 1 << 26, g_dtype="bf16"), 50, "Adam, bf16 grads, 2^26"),
+        "adam26_bf16param": (lambda d: case_adam(d, 1 << 26, p_dtype="bf16"), 50, "Adam, bf16 params, 2^26"),
+        "adam26_coupled_l2": (lambda d: case_adam(d, 1 << 26, flags=BC), 50, "Adam, coupled L2 decay (IEEE parameter path), 2^26"),
         "adam_bf16grad": (lambda d: case_adam(d, 1 << 28, g_dtype="bf16"), 50, "Adam, bf16 grads, 2^28"),
         "adam_bf16param": (lambda d: case_adam(d, 1 << 28, p_dtype="bf16"), 50, "Adam, bf16 params, fp32 grads, 2^28"),
         "adam_bf16both": (lambda d: case_adam(d, 1 << 28, g_dtype="bf16", p_dtype="bf16"), 50, "Adam, bf16 params and grads, 2^28"),
