@@ -131,6 +131,18 @@ int dt8_selfcheck_divide(const float *s, const float *N, int64_t n, float *out, 
  */
 int dt8_selfcheck_divide_const(const float *s, float d, int64_t n, float *out, void *stream);
 
+/*
+ * Diagnostics, host only.  The kernels keep their encode tables at fixed shared-memory addresses
+ * (the table of bucket key k at byte 4*k, the unsigned one shifted below the signed one), so a
+ * table set must fit between the reduction scratch and the decode tables without overlap; the
+ * library checks that once per device and answers DT8_ERR_UNSUPPORTED otherwise.
+ * dt8_selfcheck_table_extents writes the first bucket key and the number of entries of this
+ * build's signed and unsigned encode tables; dt8_selfcheck_layout_fits answers 1 if tables of the
+ * given extents fit the layout and 0 if not (a test can so see the check refuse).
+ */
+int dt8_selfcheck_table_extents(uint32_t *s_first, int *s_entries, uint32_t *u_first, int *u_entries);
+int dt8_selfcheck_layout_fits(uint32_t s_first, int s_entries, uint32_t u_first, int u_entries);
+
 /* Optional: upload the constant tables to the current device now (otherwise the first call does
  * it).  Blocking; call outside stream capture. */
 int dt8_init(void);

@@ -41,6 +41,7 @@ EXPORTS = (
     "dt8_dequantize_blockwise", "dt8_sgd_step",
     "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
     "dt8_sgd_step_ex", "dt8_adam_step_ex", "dt8_sgd_step_multi_ex", "dt8_adam_step_multi_ex",
+    "dt8_selfcheck_table_extents", "dt8_selfcheck_layout_fits",
 )
 
 
@@ -78,6 +79,8 @@ def load_library() -> ctypes.CDLL:
     lib.dt8_selfcheck_encode_host.argtypes = [i32, vp, i64, vp]
     lib.dt8_selfcheck_divide.argtypes = [vp, vp, i64, vp, vp]
     lib.dt8_selfcheck_divide_const.argtypes = [vp, f32, i64, vp, vp]
+    lib.dt8_selfcheck_table_extents.argtypes = [vp, vp, vp, vp]
+    lib.dt8_selfcheck_layout_fits.argtypes = [u32, i32, u32, i32]
     lib.dt8_init.argtypes = []
     lib.dt8_quantize_blockwise.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     lib.dt8_dequantize_blockwise.argtypes = [vp, vp, i64, i32, i32, vp, vp]

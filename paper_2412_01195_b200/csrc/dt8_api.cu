@@ -318,6 +318,26 @@ int dt8_selfcheck_encode_host(int is_signed, const float* v_host, int64_t n, uin
 }
 
 
+int dt8_selfcheck_layout_fits(uint32_t s_first, int s_entries, uint32_t u_first, int u_entries) {
+  if (s_entries < 1 || u_entries < 1 || s_first < 1 || u_first < 1) return 0;
+  EncMeta em;
+  em.s_first = s_first;
+  em.u_first = u_first;
+  em.s_n = s_entries;
+  em.u_n = u_entries;
+  return layout_ok(em) ? 1 : 0;
+}
+
+int dt8_selfcheck_table_extents(uint32_t* s_first, int* s_entries, uint32_t* u_first, int* u_entries) {
+  const Tables* ht = host_tables();
+  if (!ht || !s_first || !s_entries || !u_first || !u_entries) return DT8_ERR_INVALID_ARG;
+  *s_first = ht->enc_signed.first_key;
+  *s_entries = ht->enc_signed.num_entries;
+  *u_first = ht->enc_unsigned.first_key;
+  *u_entries = ht->enc_unsigned.num_entries;
+  return DT8_OK;
+}
+
 int dt8_init(void) {
   LaunchCtx ctx;
   return ensure_device(&ctx, nullptr);

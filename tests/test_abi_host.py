@@ -114,6 +114,22 @@ def test_table_encoder_strided_sweep_of_all_floats(signed):
         assert np.array_equal(dt8.dt8_selfcheck_encode_host(signed, v), oracle.nearest(Q, v))
 
 
+def test_shared_memory_layout_check_accepts_this_build_and_refuses_tables_that_do_not_fit(lib):
+    """The kernels address their tables at fixed shared-memory offsets; the host check that
+    guards this must pass for the tables of the build and fail for doctored extents."""
+    sf, sn, uf, un = ctypes.c_uint32(), ctypes.c_int(), ctypes.c_uint32(), ctypes.c_int()
+    assert lib.dt8_selfcheck_table_extents(ctypes.byref(sf), ctypes.byref(sn), ctypes.byref(uf),
+                                           ctypes.byref(un)) == dt8.DT8_OK
+    fits = lambda a, b, c, d: lib.dt8_selfcheck_layout_fits(a, b, c, d)
+    assert fits(sf.value, sn.value, uf.value, un.value) == 1
+    assert fits(sf.value, sn.value + 4096, uf.value, un.value) == 0      # signed table runs into the decode tables
+    assert fits(sf.value, sn.value, uf.value, un.value + 4096) == 0      # unsigned table runs into the signed one
+    assert fits(sf.value, sn.value, uf.value - 8192, un.value) == 0      # unsigned table starts below the scratch
+    assert fits(sf.value - 4096, sn.value, uf.value, un.value) == 0      # signed table overlaps the unsigned one
+    assert fits(0, 1, 0, 1) == 0 and fits(sf.value, 0, uf.value, un.value) == 0
+    assert lib.dt8_selfcheck_table_extents(None, None, None, None) == dt8.DT8_ERR_INVALID_ARG
+
+
 def test_non_finite_inputs_stay_inside_the_tables():
     v = np.array([np.nan, -np.nan, np.inf, -np.inf, 3e38, -3e38], np.float32)
     for signed in (True, False):

@@ -251,3 +251,50 @@ def test_the_benchmark_loop_on_sampled_blocks():
     assert_codes_match(to_np(mc)[idx], s_ref[0])
     assert_codes_match(to_np(rc)[idx], s_ref[2])
     assert_params_close(to_np(w)[idx], w_ref, 1e-6)
+
+
+# ------------------------------------------------------------------------------------------------
+# the constant-divisor division of the IEEE Adam update
+# ------------------------------------------------------------------------------------------------
+def test_division_by_the_bias_corrections_is_correctly_rounded():
+    """m'/(1 - beta1^t) and r'/(1 - beta2^t) use a host-made reciprocal and a residual correction
+    instead of the IEEE division.  For every divisor of that form that a run can meet -- beta 0.9
+    (t up to where 1 - beta^t rounds to 1), beta 0.999 (t = 1 .. 2000 and 200 steps spread up to
+    1e6), a few other betas, and 1 (no bias correction) -- the routine must return the correctly
+    rounded quotient: all 2^23 mantissas of the dividend in two binades for a sample of the
+    divisors, 2^18 random dividends for each of the others, plus dividends outside the fast range
+    (zero, tiny, huge), which take the IEEE division.  The reference is the binary64 quotient
+    rounded once (a quotient of two binary32 numbers is never a binary32 rounding boundary)."""
+    def bc(beta, t):
+        return float(np.float32(1.0 - float(np.float32(beta)) ** t))
+    divisors = {1.0}
+    for t in range(1, 200):
+        divisors.add(bc(0.9, t))
+    for t in list(range(1, 2001)) + [int(v) for v in np.logspace(3.3, 6, 200)]:
+        divisors.add(bc(0.999, t))
+    for beta in (0.5, 0.8, 0.95, 0.98, 0.99, 0.9999):
+        for t in (1, 2, 3, 10, 100, 1000):
+            divisors.add(bc(beta, t))
+    divisors = sorted(d for d in divisors if d > 0)
+    assert len(divisors) > 2000
+    gen = torch.Generator(device=DEV).manual_seed(77)
+    man = torch.arange(1 << 23, dtype=torch.int32, device=DEV)
+    full = torch.cat([(man | 0x3F800000).view(torch.float32), (man | 0x40000000).view(torch.float32)])
+    rnd_bits = torch.randint(0, 1 << 23, (1 << 18,), generator=gen, device=DEV, dtype=torch.int32)
+    expo = torch.randint(90, 160, (1 << 18,), generator=gen, device=DEV, dtype=torch.int32) << 23
+    sign = torch.randint(0, 2, (1 << 18,), generator=gen, device=DEV, dtype=torch.int32) << 31
+    rnd = (rnd_bits | expo | sign).view(torch.float32)
+    edge = torch.tensor([0.0, -0.0, 1e-30, -1e-30, 1e-38, 1e-42, 3e38, -3e38, 2.0 ** -60, 2.0 ** 60,
+                         2.0 ** -61, 2.0 ** 61], device=DEV)
+    rnd = torch.cat([rnd, edge])
+    out_full, out_rnd = torch.empty_like(full), torch.empty_like(rnd)
+    for i, d in enumerate(divisors):
+        s, out = (full, out_full) if i % 64 == 0 else (rnd, out_rnd)
+        got = dt8.dt8_selfcheck_divide_const(s, d, out)
+        ref = (s.double() / d).float()
+        bad = torch.nonzero(got.view(torch.int32) != ref.view(torch.int32)).flatten()
+        assert bad.numel() == 0, (d, s[bad[:4]].tolist(), got[bad[:4]].tolist(), ref[bad[:4]].tolist())
+    # divisors outside the range of the routine take the IEEE division
+    for d in (2.0 ** -25, 3.0e7, float(np.float32(1.2e-7))):
+        got = dt8.dt8_selfcheck_divide_const(rnd, d, out_rnd)
+        assert torch.equal(got.view(torch.int32), (rnd.double() / d).float().view(torch.int32))
