@@ -252,6 +252,28 @@ def time_launches(fn, iters: int, warm: int) -> float:
     return e0.elapsed_time(e1) / iters
 
 
+def time_graph_replay(fn, reps: int = 20, iters: int = 20) -> float:
+    """Milliseconds per call of fn with the host out of the way: `reps` calls captured in a CUDA
+    graph, the graph replayed `iters` times between two events.  For launches of a few
+    microseconds the back-to-back figure of time_launches is the host's submission rate."""
+    import torch
+    fn()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(reps):
+            fn()
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (iters * reps)
+
+
 def kernel_entry(ms: float, nbytes: int, peak: float, **extra) -> dict:
     gbs = nbytes / (ms * 1e-3) / 1e9
     out = {"ms": round(ms, 5), "GBps": round(gbs, 1), "frac": round(gbs / peak, 4), "bytes_per_launch": nbytes}
@@ -437,6 +459,10 @@ def run_sub_cases(dev, names, peak):
         ms = time_launches(fn, iters, 5)
         out[name] = kernel_entry(ms, nbytes, peak, launches=iters, units=units, what=desc)
         launches += iters
+        if name.startswith("multi_"):
+            # a launch of ~20 us: also the device-side time, free of the host's submission rate
+            out[name]["ms_graph_replay"] = round(time_graph_replay(fn), 5)
+            launches += 20 * 21 + 1
         del fn
         gc.collect()
         torch.cuda.empty_cache()

@@ -111,6 +111,24 @@ def num_blocks(n: int, block_size: int) -> int:
     return (n + block_size - 1) // block_size
 
 
+class _on_device:
+    """`with torch.cuda.device(d)` only when d is not already the current device (the context
+    manager costs several microseconds per call, as much as a small launch)."""
+
+    def __init__(self, device):
+        idx = device.index if device.index is not None else torch.cuda.current_device()
+        self._guard = None if idx == torch.cuda.current_device() else torch.cuda.device(idx)
+
+    def __enter__(self):
+        if self._guard is not None:
+            self._guard.__enter__()
+
+    def __exit__(self, *exc):
+        if self._guard is not None:
+            self._guard.__exit__(*exc)
+        return False
+
+
 def _stream_ptr(stream: Optional[torch.cuda.Stream], device) -> int:
     s = stream if stream is not None else torch.cuda.current_stream(device)
     return s.cuda_stream
@@ -200,7 +218,7 @@ def dt8_selfcheck_divide(s: torch.Tensor, N: torch.Tensor, out: Optional[torch.T
     """Diagnostic: the kernels' normalising division applied to operand pairs (s_i, N_i)."""
     if out is None:
         out = torch.empty_like(s)
-    with torch.cuda.device(s.device):
+    with _on_device(s.device):
         st = load_library().dt8_selfcheck_divide(
             _dev_tensor(s, torch.float32, "s"), _dev_tensor(N, torch.float32, "N"), s.numel(),
             _dev_tensor(out, torch.float32, "out"), _stream_ptr(stream, s.device))
@@ -213,7 +231,7 @@ def dt8_selfcheck_divide_const(s: torch.Tensor, d: float, out: Optional[torch.Te
     """Diagnostic: the constant-divisor division of the IEEE Adam update applied to (s_i, d)."""
     if out is None:
         out = torch.empty_like(s)
-    with torch.cuda.device(s.device):
+    with _on_device(s.device):
         st = load_library().dt8_selfcheck_divide_const(
             _dev_tensor(s, torch.float32, "s"), float(d), s.numel(),
             _dev_tensor(out, torch.float32, "out"), _stream_ptr(stream, s.device))
@@ -239,7 +257,7 @@ def dt8_quantize_blockwise(x: torch.Tensor, block_size: int, is_signed: bool,
     if absmax is None:
         absmax = torch.empty(num_blocks(n, block_size), dtype=torch.float32, device=x.device)
     _check_layout("dt8_quantize_blockwise", n, block_size, x.device, {"codes": codes}, {"absmax": absmax})
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         st = load_library().dt8_quantize_blockwise(
             _dev_tensor(x, torch.float32, "x"), n, block_size, int(bool(is_signed)),
             _dev_tensor(codes, torch.uint8, "codes"), _dev_tensor(absmax, torch.float32, "absmax"),
@@ -254,7 +272,7 @@ def dt8_dequantize_blockwise(codes: torch.Tensor, absmax: torch.Tensor, block_si
     if out is None:
         out = torch.empty(n, dtype=torch.float32, device=codes.device)
     _check_layout("dt8_dequantize_blockwise", n, block_size, codes.device, {"out": out}, {"absmax": absmax})
-    with torch.cuda.device(codes.device):
+    with _on_device(codes.device):
         st = load_library().dt8_dequantize_blockwise(
             _dev_tensor(codes, torch.uint8, "codes"), _dev_tensor(absmax, torch.float32, "absmax"), n,
             block_size, int(bool(is_signed)), _dev_tensor(out, torch.float32, "out"),
@@ -269,7 +287,7 @@ def dt8_sgd_step(p, g, m_codes, m_absmax, lr, momentum, weight_decay, step, bloc
                   {"m_absmax": m_absmax})
     gp, gd = _grad_ptr(g)
     pp, pd = _grad_ptr(p, "p")
-    with torch.cuda.device(p.device):
+    with _on_device(p.device):
         st = load_library().dt8_sgd_step_ex(
             pp, pd, gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
             _dev_tensor(m_absmax, torch.float32, "m_absmax"), p.numel(), lr, momentum, weight_decay,
@@ -284,7 +302,7 @@ def dt8_adam_step(p, g, m_codes, m_absmax, r_codes, r_absmax, lr, beta1, beta2, 
                   {"m_absmax": m_absmax, "r_absmax": r_absmax})
     gp, gd = _grad_ptr(g)
     pp, pd = _grad_ptr(p, "p")
-    with torch.cuda.device(p.device):
+    with _on_device(p.device):
         st = load_library().dt8_adam_step_ex(
             pp, pd, gp, gd, _dev_tensor(m_codes, torch.uint8, "m_codes"),
             _dev_tensor(m_absmax, torch.float32, "m_absmax"), _dev_tensor(r_codes, torch.uint8, "r_codes"),
@@ -356,7 +374,7 @@ def dt8_sgd_step_multi(ps, gs, m_codes, m_absmax, lr, momentum, weight_decay, st
     pl = _TypedPtrList(ps, "p")
     mc = _PtrList(m_codes, torch.uint8, "m_codes")
     ma = _PtrList(m_absmax, torch.float32, "m_absmax")
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         st = load_library().dt8_sgd_step_multi_ex(
             len(ps), pl.ptr, pl.dtype, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr,
             ctypes.cast(narr, ctypes.c_void_p), lr, momentum, weight_decay, step, block_size,
@@ -375,7 +393,7 @@ def dt8_adam_step_multi(ps, gs, m_codes, m_absmax, r_codes, r_absmax, lr, beta1,
     ma = _PtrList(m_absmax, torch.float32, "m_absmax")
     rc = _PtrList(r_codes, torch.uint8, "r_codes")
     ra = _PtrList(r_absmax, torch.float32, "r_absmax")
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         st = load_library().dt8_adam_step_multi_ex(
             len(ps), pl.ptr, pl.dtype, ctypes.cast(garr, ctypes.c_void_p), gd, mc.ptr, ma.ptr, rc.ptr, ra.ptr,
             ctypes.cast(narr, ctypes.c_void_p), lr, beta1, beta2, eps, weight_decay, step, block_size,
@@ -418,7 +436,7 @@ class PreparedTensorList:
 
     def sgd_step(self, lr, momentum, weight_decay, step, block_size=2048, stream=None) -> None:
         self._check_block_size("PreparedTensorList.sgd_step", block_size)
-        with torch.cuda.device(self.device):
+        with _on_device(self.device):
             st = load_library().dt8_sgd_step_multi_ex(
                 self.num, self._p.ptr, self._p.dtype, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
                 self._mc.ptr, self._ma.ptr, ctypes.cast(self._n, ctypes.c_void_p), lr, momentum,
@@ -430,7 +448,7 @@ class PreparedTensorList:
         if self._rc is None or self._ra is None:
             raise ValueError("this list was prepared without second-moment states")
         self._check_block_size("PreparedTensorList.adam_step", block_size)
-        with torch.cuda.device(self.device):
+        with _on_device(self.device):
             st = load_library().dt8_adam_step_multi_ex(
                 self.num, self._p.ptr, self._p.dtype, ctypes.cast(self._g, ctypes.c_void_p), self.g_dtype,
                 self._mc.ptr, self._ma.ptr, self._rc.ptr, self._ra.ptr,

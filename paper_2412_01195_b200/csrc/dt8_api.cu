@@ -91,6 +91,20 @@ int ensure_device(LaunchCtx* ctx, void* stream) {
       std::memset(staging.enc_u, 0, sizeof(staging.enc_u));
       std::memcpy(staging.enc_s, ht->enc_signed.entries, sizeof(uint32_t) * ht->enc_signed.num_entries);
       std::memcpy(staging.enc_u, ht->enc_unsigned.entries, sizeof(uint32_t) * ht->enc_unsigned.num_entries);
+      // the shared-memory image of the step kernels: encode tables at their byte addresses (the
+      // unsigned one shifted by kEncUOffset), decode tables replicated once per lane
+      std::memset(staging.image, 0, sizeof(staging.image));
+      if (layout_ok(em)) {
+        const EncBounds bs = make_bounds(em.s_first, em.s_n), bu = make_bounds(em.u_first, em.u_n);
+        uint32_t* img = staging.image;
+        for (int i = 0; i < em.s_n; ++i) img[(bs.lo4 - kImageBase) / 4 + i] = staging.enc_s[i];
+        for (int i = 0; i < em.u_n; ++i)
+          img[(static_cast<int64_t>(bu.lo4) + kEncUOffset - kImageBase) / 4 + i] = staging.enc_u[i];
+        for (int i = 0; i < 256 * 64; ++i) {   // code = i / 64, table = (i / 32) % 2, lane = i % 32
+          const float v = (i & 32) ? staging.dec_u[i >> 6] : staging.dec_s[i >> 6];
+          std::memcpy(&img[(kDecodeAddr - kImageBase) / 4 + i], &v, 4);
+        }
+      }
       e = cudaMemcpyToSymbol(g_tables, &staging, sizeof(staging));
       if (e != cudaSuccess) return cuda_fail(e);
       void* addr = nullptr;

@@ -19,7 +19,7 @@ from typing import Optional, Sequence
 
 import torch
 
-from . import DT8Error, DT8_OK, _stream_ptr, load_library
+from . import DT8Error, DT8_OK, _on_device, _stream_ptr, load_library
 
 __all__ = ["dt8_rev_coupling_forward", "dt8_rev_coupling_inverse", "dt8_rev_space_to_depth",
            "dt8_rev_depth_to_space", "rev_block_forward", "rev_block_inverse", "rev_block_backward",
@@ -67,7 +67,7 @@ def _couple(fn_name: str, a: torch.Tensor, t: torch.Tensor, out: torch.Tensor, w
     if out.shape != a.shape or t.numel() != n * half or t.device != a.device or out.device != a.device:
         raise ValueError(f"{fn_name}: out must have the activation's shape and t half of its elements, "
                          "all on one device")
-    with torch.cuda.device(a.device):
+    with _on_device(a.device):
         st = getattr(_lib(), fn_name)(_act(a, "activation"), _act(t, "t"), _act(out, "out"), n, half,
                                       int(which), _stream_ptr(stream, a.device))
     _check(st, fn_name)
@@ -92,7 +92,7 @@ def dt8_rev_space_to_depth(x: torch.Tensor, out: Optional[torch.Tensor] = None, 
         out = torch.empty((n, 4 * c, f // 2, t // 2), dtype=torch.float32, device=x.device)
     if out.numel() != x.numel() or out.device != x.device:
         raise ValueError("dt8_rev_space_to_depth: out must hold as many elements as x, on its device")
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         st = _lib().dt8_rev_space_to_depth(_act(x, "x"), n, c, f, t, _act(out, "out"),
                                            _stream_ptr(stream, x.device))
     _check(st, "dt8_rev_space_to_depth")
@@ -108,7 +108,7 @@ def dt8_rev_depth_to_space(y: torch.Tensor, out: Optional[torch.Tensor] = None, 
         out = torch.empty((n, c4 // 4, 2 * fo, 2 * to), dtype=torch.float32, device=y.device)
     if out.numel() != y.numel() or out.device != y.device:
         raise ValueError("dt8_rev_depth_to_space: out must hold as many elements as y, on its device")
-    with torch.cuda.device(y.device):
+    with _on_device(y.device):
         st = _lib().dt8_rev_depth_to_space(_act(y, "y"), n, c4 // 4, fo, to, _act(out, "out"),
                                            _stream_ptr(stream, y.device))
     _check(st, "dt8_rev_depth_to_space")
