@@ -205,3 +205,39 @@ def test_rev_sequence_trains_like_the_stored_activation_network():
     # inference path keeps no graph
     with torch.no_grad():
         assert _rel(net(x), h) < 1e-5
+
+
+# ------------------------------------------------------------------------------------------------
+# the benchmark's shapes: the checker on sampled samples, a library identity on everything
+# ------------------------------------------------------------------------------------------------
+def test_benchmark_shapes_sampled_against_the_checker():
+    """128 activations of the first reversible stage (48 x 80 x 200), as bench.py times them.  The
+    checker follows samples 0, 77 and 127 (samples are independent); on all samples the coupling
+    equals torch's element-wise add / subtract (one IEEE operation per element on both sides) and
+    the rearrangement equals torch's pixel_unshuffle of the row-major reading."""
+    n, c, f, t = 128, 48, 80, 200
+    x = synth.normal(n * c * f * t, 1.0, 31, device=DEV).reshape(n, c, f, t)
+    br = synth.normal(n * c * f * t // 2, 1.0, 32, device=DEV).reshape(n, c // 2, f, t)
+    picks = [0, 77, 127]
+    for which in (0, 1):
+        lo, hi = (0, c // 2) if which == 0 else (c // 2, c)
+        y = torch.full_like(x, float("nan"))
+        rev.dt8_rev_coupling_forward(x, br, y, which)
+        assert torch.equal(y[:, lo:hi], x[:, lo:hi] + br)
+        want = np.full((len(picks), c, f, t), np.nan, F32)
+        orev.couple_half(x[picks].cpu().numpy(), br[picks].cpu().numpy(), want, which, +1)
+        assert np.array_equal(y[picks].cpu().numpy().view(np.uint32), want.view(np.uint32))
+        z = torch.full_like(x, float("nan"))
+        rev.dt8_rev_coupling_inverse(y, br, z, which)
+        assert torch.equal(z[:, lo:hi], y[:, lo:hi] - br)
+        del y, z
+    del br
+    for shape in ((128, 24, 80, 200), (512, 75, 20, 50)):
+        n, c, f, t = shape
+        a = synth.normal(n * c * f * t, 1.0, 33, device=DEV).reshape(shape)
+        d = rev.dt8_rev_space_to_depth(a)
+        assert torch.equal(d, torch.nn.functional.pixel_unshuffle(a, 2))
+        for k in (0, n // 2 + 1, n - 1):
+            assert np.array_equal(d[k:k + 1].cpu().numpy(), orev.space_to_depth(a[k:k + 1].cpu().numpy(), 2))
+        assert torch.equal(rev.dt8_rev_depth_to_space(d), a)
+        del a, d
