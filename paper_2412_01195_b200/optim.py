@@ -6,7 +6,9 @@ The optimizers of Section IV of the paper ("SGD (8-bit)", "Adam (8-bit)") as dro
 pointer-list entry points), whatever the number of tensors.  These classes only keep the state
 tensors and marshal pointers; all arithmetic runs in `libdt8.so`.
 
-Parameters must be contiguous fp32 CUDA tensors; gradients fp32 or bf16 (one dtype per group).
+Parameters must be contiguous fp32 or bf16 CUDA tensors (bf16 parameters are stepped without a
+32-bit copy: widened, updated in fp32, rounded once on store); gradients fp32 or bf16; one dtype
+of each per group.
 The pointer arrays are rebuilt only when a parameter's or gradient's address changes, so
 `optimizer.zero_grad(set_to_none=False)` keeps the per-step host cost at one launch.
 `state_dict()` / `load_state_dict()` carry the codes, the block maxima and the step count, so a
@@ -46,8 +48,10 @@ class _Optimizer8bit(torch.optim.Optimizer):
         for p in ps:
             if p.grad.is_sparse:
                 raise RuntimeError("sparse gradients are not supported")
-            if not (p.is_cuda and p.dtype == torch.float32 and p.is_contiguous()):
-                raise TypeError("parameters must be contiguous float32 CUDA tensors")
+            if not (p.is_cuda and p.dtype in (torch.float32, torch.bfloat16) and p.is_contiguous()):
+                raise TypeError("parameters must be contiguous float32 or bfloat16 CUDA tensors")
+        if any(p.dtype != ps[0].dtype for p in ps):
+            raise TypeError("the parameters of one group share a dtype (use one group per dtype)")
         gs = [p.grad if p.grad.is_contiguous() else p.grad.contiguous() for p in ps]
         B = group["block_size"]
         sts = [self._state_of(p, B) for p in ps]
@@ -64,19 +68,23 @@ class _Optimizer8bit(torch.optim.Optimizer):
         return cached[1]
 
     def load_state_dict(self, state_dict) -> None:
-        """torch casts every loaded state tensor to the parameter's dtype; the uint8 codes must
-        stay uint8, so they are set aside and put back untouched."""
-        codes = {}
+        """torch casts every loaded floating-point state tensor to the parameter's dtype and
+        leaves the others alone only by their dtype; the uint8 codes must stay uint8 and the
+        block maxima fp32 (also under bf16 parameters), so both are set aside and put back
+        untouched."""
+        keep = ("_codes", "_absmax")
+        held = {}
         stripped = {"param_groups": state_dict["param_groups"], "state": {}}
         for pid, st in state_dict["state"].items():
-            stripped["state"][pid] = {k: v for k, v in st.items() if not k.endswith("_codes")}
-            codes[pid] = {k: v for k, v in st.items() if k.endswith("_codes")}
+            stripped["state"][pid] = {k: v for k, v in st.items() if not k.endswith(keep)}
+            held[pid] = {k: v for k, v in st.items() if k.endswith(keep)}
         super().load_state_dict(stripped)
         ids = [pid for g in state_dict["param_groups"] for pid in g["params"]]
         params = [p for g in self.param_groups for p in g["params"]]
         for pid, p in zip(ids, params):
-            for k, v in codes.get(pid, {}).items():
-                self.state[p][k] = v.detach().to(device=p.device, dtype=torch.uint8).clone()
+            for k, v in held.get(pid, {}).items():
+                dtype = torch.uint8 if k.endswith("_codes") else torch.float32
+                self.state[p][k] = v.detach().to(device=p.device, dtype=dtype).clone()
         # a state saved with another block size (or for another tensor) must not reach a kernel
         for group in self.param_groups:
             for p in group["params"]:

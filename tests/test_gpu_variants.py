@@ -298,3 +298,57 @@ def test_division_by_the_bias_corrections_is_correctly_rounded():
     for d in (2.0 ** -25, 3.0e7, float(np.float32(1.2e-7))):
         got = dt8.dt8_selfcheck_divide_const(rnd, d, out_rnd)
         assert torch.equal(got.view(torch.int32), (rnd.double() / d).float().view(torch.int32))
+
+
+def test_optimizer_front_end_with_bf16_parameters_steps_and_resumes():
+    """AdamW8bit on bfloat16 parameters: equal to the pointer-list entry point called by hand, and
+    a run resumed from state_dict() continues bit-identically (codes stay uint8, block maxima
+    fp32 through the round trip)."""
+    from paper_2412_01195_b200.optim import AdamW8bit
+    sizes = [(64, 33), (300,), (5, 7, 3, 3)]
+    B = 256
+
+    def params():
+        return [torch.nn.Parameter(synth.normal(int(np.prod(s)), 0.05, 2100 + i).reshape(s).to(torch.bfloat16).to(DEV))
+                for i, s in enumerate(sizes)]
+
+    def grads(step):
+        # torch wants a gradient of the parameter's dtype
+        return [synth.normal(int(np.prod(s)), 1e-2, 2200 + 10 * step + i).reshape(s).to(torch.bfloat16).to(DEV)
+                for i, s in enumerate(sizes)]
+
+    def run(ps, opt, steps):
+        for t in steps:
+            for p, g in zip(ps, grads(t)):
+                if p.grad is None:
+                    p.grad = g.clone()
+                else:
+                    p.grad.copy_(g)
+            opt.step()
+
+    pa = params()
+    oa = AdamW8bit(pa, lr=1e-3, weight_decay=0.05, block_size=B)
+    run(pa, oa, range(1, 6))
+    # by hand
+    ph = [p.detach().clone().view(-1) for p in params()]
+    sm = [dt8.new_state(p.numel(), B, True, DEV) for p in ph]
+    sr = [dt8.new_state(p.numel(), B, False, DEV) for p in ph]
+    for t in range(1, 6):
+        dt8.dt8_adam_step_multi(ph, [g.view(-1) for g in grads(t)], [s[0] for s in sm], [s[1] for s in sm],
+                                [s[0] for s in sr], [s[1] for s in sr], 1e-3, 0.9, 0.999, 1e-8, 0.05, t, B)
+    torch.cuda.synchronize()
+    for p, q in zip(pa, ph):
+        assert p.dtype == torch.bfloat16 and torch.equal(p.detach().view(-1), q)
+    # resume after 3 of the 5 steps
+    pb = params()
+    ob = AdamW8bit(pb, lr=1e-3, weight_decay=0.05, block_size=B)
+    run(pb, ob, range(1, 4))
+    sd = ob.state_dict()
+    pc = [torch.nn.Parameter(p.detach().clone()) for p in pb]
+    oc = AdamW8bit(pc, lr=1e-3, weight_decay=0.05, block_size=B)
+    oc.load_state_dict(sd)
+    assert all(st["m_codes"].dtype == torch.uint8 and st["r_absmax"].dtype == torch.float32 for st in oc.state.values())
+    run(pc, oc, range(4, 6))
+    torch.cuda.synchronize()
+    for p, q in zip(pa, pc):
+        assert torch.equal(p.detach(), q.detach())
