@@ -693,6 +693,10 @@ def run_dt8(args):
         kernels, extra = run_sub_cases(dev, DEFAULT_SUBS, peak)
         launches += extra
         rev_memory = run_rev_memory(dev)
+        # the same at two other depths: the reversible figure does not depend on the depth
+        rev_memory["by_depth"] = [{k: m[k] for k in ("blocks", "reversible_bytes_per_sample", "stored_bytes_per_sample",
+                                                     "memory_ratio", "time_ratio")}
+                                  for m in (run_rev_memory(dev, blocks=4), run_rev_memory(dev, blocks=16))]
 
     out = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world,
