@@ -448,7 +448,9 @@ def sub_cases():
     return c
 
 
-def run_sub_cases(dev, names, peak):
+def run_sub_cases(dev, names, peak, clock_of=None):
+    """Times the named cases; clock_of = (gpu index, uuid) also samples the SM clock during each
+    case (the cases that are bound by instruction issue depend on it)."""
     import gc
     import torch
     cases = sub_cases()
@@ -456,8 +458,17 @@ def run_sub_cases(dev, names, peak):
     for name in names:
         build, iters, desc = cases[name]
         fn, nbytes, units = build(dev)
+        sampler = None
+        if clock_of is not None:
+            time_launches(fn, 5, 0)
+            sampler = ClockSampler(clock_of[0], clock_of[1], period_s=0.002)
+            sampler.start()
         ms = time_launches(fn, iters, 5)
         out[name] = kernel_entry(ms, nbytes, peak, launches=iters, units=units, what=desc)
+        if sampler is not None:
+            clk = sampler.stop()
+            out[name]["sm_mhz"] = clk.get("sm_mhz")
+            launches += 5
         launches += iters
         if name.startswith("multi_"):
             # a launch of ~20 us: also the device-side time, free of the host's submission rate
@@ -618,7 +629,7 @@ def run_dt8(args):
 
     if args.only:                              # a few sub-cases alone (what an ncu capture runs)
         names = [s for s in args.only.split(",") if s]
-        kernels, launches = run_sub_cases(dev, names, peak)
+        kernels, launches = run_sub_cases(dev, names, peak, (local_rank, uuid))
         if rank == 0:
             print(json.dumps({"only": names, "kernels": kernels, "gpu_launches": launches,
                               "peak": peak, "peak_source": peak_src}), flush=True)
@@ -690,7 +701,7 @@ def run_dt8(args):
     # ---- every other entry point, timed the same way (one GPU) ------------------------------------
     kernels, rev_memory = None, None
     if world == 1 and not args.no_kernels:
-        kernels, extra = run_sub_cases(dev, DEFAULT_SUBS, peak)
+        kernels, extra = run_sub_cases(dev, DEFAULT_SUBS, peak, (local_rank, uuid))
         launches += extra
         rev_memory = run_rev_memory(dev)
         # the same at two other depths: the reversible figure does not depend on the depth

@@ -45,7 +45,8 @@ divide_const_kernel(const float* __restrict__ s, ConstDivisor cd, float* __restr
   {
     const float a = fabsf(s[i]);
     const bool fast = cd.usable && a >= kConstDivMinDividend && a <= kConstDivMaxDividend;
-    out[i] = fast ? cd.div<true>(s[i]) : cd.div<false>(s[i]);
+    // the packed form the step kernel uses (both lanes carry the same dividend here)
+    out[i] = fast ? lo2(cd.div2<true>(pack2(s[i], s[i]))) : cd.div<false>(s[i]);
   }
 }
 
