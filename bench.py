@@ -545,7 +545,8 @@ def run_rev_memory(dev, blocks: int = 8, batch: int = 8, channels: int = 48, fre
                                    torch.nn.Conv2d(c, c, 3, padding=1))
     torch.manual_seed(0)
     net = rev.RevSequence([rev.RevBlock(branch(), branch()) for _ in range(blocks)]).to(dev)
-    x = torch.randn(batch, channels, freq, frames, device=dev)
+    from paper_2412_01195_b200 import synth
+    x = synth.normal(batch * channels * freq * frames, 1.0, 41, device=dev).reshape(batch, channels, freq, frames)
     c = channels // 2
 
     def stored(inp):
