@@ -83,7 +83,7 @@ def test_coupling_argument_checks():
 # invertible down-sampling (Eq. revnet6, r = 2)
 # ------------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("shape", [(1, 1, 2, 2), (1, 2, 2, 4), (2, 3, 4, 6), (3, 5, 6, 10), (2, 24, 80, 200),
-                                   (2, 48, 40, 100), (3, 75, 20, 50), (1, 7, 2, 2050), (4, 1, 34, 4), (2, 2, 126, 102), (5, 3, 2, 6142)])
+                                   (2, 48, 40, 100), (3, 75, 20, 50), (1, 7, 2, 2050), (4, 1, 34, 4), (2, 2, 126, 102), (5, 3, 2, 6142), (3, 2, 3070, 2), (2, 5, 2, 2)])
 def test_space_to_depth_and_back_match_the_checker(shape):
     x = torch.arange(int(np.prod(shape)), dtype=torch.float32).reshape(shape) * 0.5 - 7
     y = rev.dt8_rev_space_to_depth(x.to(DEV))
