@@ -98,7 +98,7 @@ int launch_coupling(const float* in, const float* t, float* out, int64_t batch, 
 // invertible down-sampling, r = 2.  In the N x C x F x T layout the two input rows 2fo, 2fo + 1 of
 // a channel are adjacent, and the four output channels of an input channel start at the same
 // offset as the input channel itself (4 * Fo * To == F * T).  A thread takes VEC consecutive
-// elements of one input row (VEC = 4, or 2 when T is not a multiple of 4): the even ones go to
+// elements of one input row (VEC = 8, 4 or 2, the largest that divides T): the even ones go to
 // output channel 2 df, the odd ones to 2 df + 1, at column (t / 2) of row fo.  Consecutive threads
 // take consecutive pieces of the flat input, so loads and stores are whole lines per warp.
 // ---------------------------------------------------------------------------------------------
@@ -125,10 +125,42 @@ struct FastDiv {
 constexpr int kShuffleThreads = 256;
 constexpr int kShuffleUnroll = 4;
 
+// A piece: VEC consecutive elements of a flat row (In) and the VEC / 2 even or odd ones (Out).
+struct Float8 {
+  float4 a, b;
+};
 template <int VEC> struct Piece;
+template <> struct Piece<8> {
+  typedef Float8 In;
+  typedef float4 Out;
+  static __device__ __forceinline__ In load_in(const float* p) {
+    In v;
+    v.a = __ldcs(reinterpret_cast<const float4*>(p));
+    v.b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+    return v;
+  }
+  static __device__ __forceinline__ void store_in(float* p, In v) {
+    __stcs(reinterpret_cast<float4*>(p), v.a);
+    __stcs(reinterpret_cast<float4*>(p) + 1, v.b);
+  }
+  static __device__ __forceinline__ Out load_out(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+  static __device__ __forceinline__ void store_out(float* p, Out v) { __stcs(reinterpret_cast<float4*>(p), v); }
+  static __device__ __forceinline__ Out even(In v) { return make_float4(v.a.x, v.a.z, v.b.x, v.b.z); }
+  static __device__ __forceinline__ Out odd(In v) { return make_float4(v.a.y, v.a.w, v.b.y, v.b.w); }
+  static __device__ __forceinline__ In merge(Out e, Out o) {
+    In v;
+    v.a = make_float4(e.x, o.x, e.y, o.y);
+    v.b = make_float4(e.z, o.z, e.w, o.w);
+    return v;
+  }
+};
 template <> struct Piece<4> {
   typedef float4 In;
   typedef float2 Out;
+  static __device__ __forceinline__ In load_in(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+  static __device__ __forceinline__ void store_in(float* p, In v) { __stcs(reinterpret_cast<float4*>(p), v); }
+  static __device__ __forceinline__ Out load_out(const float* p) { return __ldcs(reinterpret_cast<const float2*>(p)); }
+  static __device__ __forceinline__ void store_out(float* p, Out v) { __stcs(reinterpret_cast<float2*>(p), v); }
   static __device__ __forceinline__ Out even(In v) { return make_float2(v.x, v.z); }
   static __device__ __forceinline__ Out odd(In v) { return make_float2(v.y, v.w); }
   static __device__ __forceinline__ In merge(Out e, Out o) { return make_float4(e.x, o.x, e.y, o.y); }
@@ -136,6 +168,10 @@ template <> struct Piece<4> {
 template <> struct Piece<2> {
   typedef float2 In;
   typedef float Out;
+  static __device__ __forceinline__ In load_in(const float* p) { return __ldcs(reinterpret_cast<const float2*>(p)); }
+  static __device__ __forceinline__ void store_in(float* p, In v) { __stcs(reinterpret_cast<float2*>(p), v); }
+  static __device__ __forceinline__ Out load_out(const float* p) { return __ldcs(p); }
+  static __device__ __forceinline__ void store_out(float* p, Out v) { __stcs(p, v); }
   static __device__ __forceinline__ Out even(In v) { return v.x; }
   static __device__ __forceinline__ Out odd(In v) { return v.y; }
   static __device__ __forceinline__ In merge(Out e, Out o) { return make_float2(e, o); }
@@ -177,10 +213,10 @@ shuffle_kernel(const float* __restrict__ src, float* __restrict__ dst, uint32_t 
       if (i < pieces) {
         off[k] = map.deep_offset<VEC>(i);
         if (TO_DEPTH) {
-          flat[k] = __ldcs(reinterpret_cast<const typename P::In*>(src) + i);
+          flat[k] = P::load_in(src + static_cast<int64_t>(i) * VEC);
         } else {
-          ev[k] = __ldcs(reinterpret_cast<const typename P::Out*>(src + off[k]));
-          od[k] = __ldcs(reinterpret_cast<const typename P::Out*>(src + off[k] + chan_stride));
+          ev[k] = P::load_out(src + off[k]);
+          od[k] = P::load_out(src + off[k] + chan_stride);
         }
       }
     }
@@ -189,10 +225,10 @@ shuffle_kernel(const float* __restrict__ src, float* __restrict__ dst, uint32_t 
       const uint32_t i = base + k * kShuffleThreads + threadIdx.x;
       if (i < pieces) {
         if (TO_DEPTH) {
-          __stcs(reinterpret_cast<typename P::Out*>(dst + off[k]), P::even(flat[k]));
-          __stcs(reinterpret_cast<typename P::Out*>(dst + off[k] + chan_stride), P::odd(flat[k]));
+          P::store_out(dst + off[k], P::even(flat[k]));
+          P::store_out(dst + off[k] + chan_stride, P::odd(flat[k]));
         } else {
-          __stcs(reinterpret_cast<typename P::In*>(dst) + i, P::merge(ev[k], od[k]));
+          P::store_in(dst + static_cast<int64_t>(i) * VEC, P::merge(ev[k], od[k]));
         }
       }
     }
@@ -292,9 +328,10 @@ int launch_shuffle(const float* src, float* dst, int64_t N, int64_t C, int64_t F
   const float* flat = TO_DEPTH ? src : dst;
   const float* deep = TO_DEPTH ? dst : src;
   // 16-byte pieces need rows of a multiple of 4 floats (then output rows are a multiple of 2)
-  const bool vec4 = (T % 4 == 0) && aligned_to(flat, 16) && aligned_to(deep, 8);
+  const bool vec8 = (T % 8 == 0) && aligned_to(flat, 16) && aligned_to(deep, 16);
+  const bool vec4 = vec8 || ((T % 4 == 0) && aligned_to(flat, 16) && aligned_to(deep, 8));
   if (!vec4 && !(aligned_to(flat, 8) && aligned_to(deep, 4))) return DT8_ERR_ALIGNMENT;
-  const int vec = vec4 ? 4 : 2;
+  const int vec = vec8 ? 8 : vec4 ? 4 : 2;
   const int64_t pieces = total / vec;
   if (pieces >= (int64_t(1) << 31) || N * C * F >= (int64_t(1) << 32)) return DT8_ERR_UNSUPPORTED;
   int dev = 0, sms = 0;
@@ -325,7 +362,9 @@ int launch_shuffle(const float* src, float* dst, int64_t N, int64_t C, int64_t F
   const int64_t want = (pieces + tile - 1) / tile;
   const int64_t cap = static_cast<int64_t>(sms) * 16;
   const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
-  if (vec4)
+  if (vec8)
+    shuffle_kernel<8, TO_DEPTH><<<grid, kShuffleThreads, 0, s>>>(src, dst, static_cast<uint32_t>(pieces), map);
+  else if (vec4)
     shuffle_kernel<4, TO_DEPTH><<<grid, kShuffleThreads, 0, s>>>(src, dst, static_cast<uint32_t>(pieces), map);
   else
     shuffle_kernel<2, TO_DEPTH><<<grid, kShuffleThreads, 0, s>>>(src, dst, static_cast<uint32_t>(pieces), map);
