@@ -230,6 +230,7 @@ AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float w
   h.rbc1 = d1.rd;
   h.rbc2 = d2.rd;
   h.const_div = (d1.usable && d2.usable) ? 1 : 0;
+  h.neg_zero = -0.0f;
   return h;
 }
 
@@ -430,7 +431,7 @@ int dt8_sgd_step_ex(void* p, int p_dtype, const void* g, int g_dtype, uint8_t* m
   LaunchCtx ctx;
   rc = ensure_device(&ctx, stream);
   if (rc != DT8_OK) return rc;
-  const SgdHyper h{lr, momentum, weight_decay};
+  const SgdHyper h{lr, momentum, weight_decay, -0.0f};
   return launch_sgd(a, a.nb, block_size, p_dtype, g_dtype, h, ctx);
 }
 
@@ -532,7 +533,7 @@ int dt8_sgd_step_multi_ex(int num_tensors, void* const* p, int p_dtype, const vo
                           const int64_t* n, float lr, float momentum, float weight_decay,
                           int64_t step, int block_size, void* stream) {
   if (step < 1 || !sgd_hyper_ok(lr, momentum, weight_decay)) return DT8_ERR_INVALID_ARG;
-  const SgdHyper h{lr, momentum, weight_decay};
+  const SgdHyper h{lr, momentum, weight_decay, -0.0f};
   return run_multi(num_tensors, p, p_dtype, g, g_dtype, m_codes, m_absmax, nullptr, nullptr, n,
                    block_size, false, stream,
                    [&](const MultiArgs& a, int64_t blocks, const LaunchCtx& ctx) {

@@ -55,26 +55,26 @@ bool build_enc(int W, int shift, EncTable* t) {
   const bool is_signed = (W == 7);
   if (is_signed ? shift != 16 : shift != 15) return false;
   // field layouts, see dt8_tables.h
-  const uint32_t ones = is_signed ? 0x7F00u : 0x1FF00u;
+  const uint32_t ones = is_signed ? 0x7F00u : 0u;   // the bits between the count and the field
   const int field_shift = is_signed ? 15 : 17;
   const uint32_t none = (is_signed ? 0x1FFFFu : 0x7FFFu) << field_shift;
   t->num_entries = n;
-  t->entries[0] = 0u | ones | none;
+  t->entries[0] = 1u | ones | none;   // the count is stored plus one
   int next = 0;  // first threshold not yet below the current bucket
   for (int idx = 1; idx <= n - 2; ++idx) {
     const uint32_t start = (t->first_key + static_cast<uint32_t>(idx - 1)) << shift;
     const uint32_t end = start + (1u << shift);
     while (next < P && thr_bits[next] < start) ++next;
-    uint32_t entry = static_cast<uint32_t>(next) | ones | none;
+    uint32_t entry = static_cast<uint32_t>(next + 1) | ones | none;
     if (next < P && thr_bits[next] < end) {
       if (next + 1 < P && thr_bits[next + 1] < end) return false;  // two thresholds in a bucket
       const uint32_t low = thr_bits[next] - start;
       const uint32_t field = is_signed ? 2u * low + (thr_exact[next] ? 0u : 1u) : low;
-      entry = static_cast<uint32_t>(next) | ones | (field << field_shift);
+      entry = static_cast<uint32_t>(next + 1) | ones | (field << field_shift);
     }
     t->entries[idx] = entry;
   }
-  t->entries[n - 1] = static_cast<uint32_t>(P) | ones | none;
+  t->entries[n - 1] = static_cast<uint32_t>(P + 1) | ones | none;
   return true;
 }
 

@@ -29,11 +29,15 @@ constexpr int kSignedShift = 16;    // 7 mantissa bits per bucket: width <= 2^-7
 constexpr int kUnsignedShift = 15;  // 8 mantissa bits per bucket
 constexpr int kMaxEncEntries = 6656;
 
-// Entry layouts (low byte = number of thresholds below the bucket, i.e. the magnitude pattern at
-// the bucket's lower edge; the bits between it and the threshold field are all ones so that the
-// compare below is decided by the threshold field alone):
-//   signed   : T2 << 15 | 0x7F00 | count,  T2 = 2*threshold_low16 + (tie flag ? 0 : 1), 17 bits
-//   unsigned : thr << 17 | 0x1FF00 | count, thr = threshold_low15
+// Entry layouts.  The low bits hold one more than the number of thresholds below the bucket (the
+// magnitude pattern at the bucket's lower edge, plus one), the top bits the threshold field:
+//   signed   : T2 << 15 | 0x7F00 | (count + 1),  T2 = 2*threshold_low16 + (tie flag ? 0 : 1), 17 bits
+//   unsigned : thr << 17 | (count + 1),           thr = threshold_low15, count + 1 in 9 bits
+// A query word x carries its own threshold field in the same place, and the look-up returns
+// entry - (x < entry ? 1 : 0): the pattern is count when the query's field does not exceed the
+// stored one and count + 1 when it does.  The bits of an entry below its threshold field are never
+// smaller than a query's (signed: ones down to the byte, above every bucket key up to 1.0;
+// unsigned: the query has zeros there and count + 1 >= 1), so equal fields compare as "not above".
 // A bucket without a threshold stores the all-ones field, which no query exceeds.
 struct EncTable {
   int shift;            // bucket key = bits(a) >> shift
@@ -80,6 +84,18 @@ DT8_HD uint32_t byte_perm(uint32_t x, uint32_t y, uint32_t sel) {
 #endif
 }
 
+// entry - (x < entry ? 1 : 0).  On the device the borrow of x - entry is taken off the entry
+// (sub.cc / subc): two instructions, no predicate and no select.
+DT8_HD uint32_t below_by_borrow(uint32_t entry, uint32_t x) {
+#if defined(__CUDA_ARCH__)
+  uint32_t diff, r;
+  asm("{\n\tsub.cc.u32 %0, %3, %2;\n\tsubc.u32 %1, %2, 0;\n\t}" : "=r"(diff), "=r"(r) : "r"(entry), "r"(x));
+  return r;
+#else
+  return entry - (x < entry ? 1u : 0u);
+#endif
+}
+
 // Bounds of one encode table in "byte address" form: bucket key k is looked up at byte offset
 // 4*k.  lo4 = 4*(first_key - 1) is the entry "everything below", hi4 the entry "a >= 1".  In the
 // kernels the table is placed in shared memory so that 4*k IS the shared-memory address of the
@@ -113,7 +129,7 @@ DT8_HD uint32_t lookup_signed(const Fetch& fetch, const EncBounds& t, uint32_t v
   k4 = k4 < t.lo4 ? t.lo4 : k4;
   if (CLAMP_HI) k4 = k4 > t.hi4 ? t.hi4 : k4;
   const uint32_t e = fetch(k4);
-  return e + (x > e ? 1u : 0u);
+  return below_by_borrow(e, x);
 }
 
 // Unsigned table; negative values (and -0) count as 0.  lo4 << 13 is the bit pattern of the
@@ -128,7 +144,7 @@ DT8_HD uint32_t lookup_unsigned(const Fetch& fetch, const EncBounds& t, uint32_t
   uint32_t k4 = (a >> 13) & 0x7FFFCu;
   if (CLAMP_HI) k4 = k4 > t.hi4 ? t.hi4 : k4;
   const uint32_t e = fetch(k4);
-  return e + ((a << 17) > e ? 1u : 0u);
+  return below_by_borrow(e, a << 17);
 }
 
 // Gathers the low bytes of four words into one word (word 0 in byte 0).
