@@ -120,6 +120,16 @@ int dt8_selfcheck_encode_host(int is_signed, const float *v_host, int64_t n, uin
 int dt8_selfcheck_divide(const float *s, const float *N, int64_t n, float *out, void *stream);
 
 /*
+ * Diagnostic, device: out_i = the reciprocal of N_i that the routine above starts from (Eq. quant1:
+ * one reciprocal per block, then one multiply and two fused multiply-adds per element).  The
+ * residual correction is exact only when that reciprocal is the correctly rounded one, so a test
+ * checks it for every binary32 mantissa.  out_i = 0 where the routine takes the IEEE division
+ * instead (N_i = 0 included).  No step, quantize or dequantize call uses it.
+ *   N  device, const float[n];   out  device, float[n]
+ */
+int dt8_selfcheck_reciprocal(const float *N, int64_t n, float *out, void *stream);
+
+/*
  * Diagnostic, device: out_i = s_i / d computed by the routine the IEEE form of the Adam parameter
  * update uses for Eq. adam's bias corrections m'/(1 - beta1^step), r'/(1 - beta2^step), whose
  * divisor is one number per launch: the host supplies the correctly rounded reciprocal of d and

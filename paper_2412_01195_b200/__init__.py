@@ -16,7 +16,7 @@ import torch
 
 __all__ = [
     "DT8Error", "lib_path", "load_library", "num_blocks",
-    "dt8_codebook", "dt8_state_bytes", "optimizer_state_bytes", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_init",
+    "dt8_codebook", "dt8_state_bytes", "optimizer_state_bytes", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_selfcheck_reciprocal", "dt8_init",
     "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step", "dt8_adam_step", "dt8_sgd_step_multi",
     "dt8_adam_step_multi", "new_state", "shard_blocks", "PreparedTensorList",
@@ -37,7 +37,8 @@ _lib = None
 EXPORTS = (
     "dt8_status_string", "dt8_last_cuda_error", "dt8_codebook", "dt8_state_bytes",
     "dt8_selfcheck_encode_host",
-    "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_init", "dt8_quantize_blockwise",
+    "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_selfcheck_reciprocal", "dt8_init",
+    "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step",
     "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
     "dt8_sgd_step_ex", "dt8_adam_step_ex", "dt8_sgd_step_multi_ex", "dt8_adam_step_multi_ex",
@@ -79,6 +80,7 @@ def load_library() -> ctypes.CDLL:
     lib.dt8_selfcheck_encode_host.argtypes = [i32, vp, i64, vp]
     lib.dt8_selfcheck_divide.argtypes = [vp, vp, i64, vp, vp]
     lib.dt8_selfcheck_divide_const.argtypes = [vp, f32, i64, vp, vp]
+    lib.dt8_selfcheck_reciprocal.argtypes = [vp, i64, vp, vp]
     lib.dt8_selfcheck_table_extents.argtypes = [vp, vp, vp, vp]
     lib.dt8_selfcheck_layout_fits.argtypes = [u32, i32, u32, i32]
     lib.dt8_init.argtypes = []
@@ -223,6 +225,19 @@ def dt8_selfcheck_divide(s: torch.Tensor, N: torch.Tensor, out: Optional[torch.T
             _dev_tensor(s, torch.float32, "s"), _dev_tensor(N, torch.float32, "N"), s.numel(),
             _dev_tensor(out, torch.float32, "out"), _stream_ptr(stream, s.device))
     _check(st, "dt8_selfcheck_divide")
+    return out
+
+
+def dt8_selfcheck_reciprocal(N: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Diagnostic: the reciprocal of N_i the normalising division starts from (0 where it takes
+    the IEEE division)."""
+    if out is None:
+        out = torch.empty_like(N)
+    with _on_device(N.device):
+        st = load_library().dt8_selfcheck_reciprocal(
+            _dev_tensor(N, torch.float32, "N"), N.numel(), _dev_tensor(out, torch.float32, "out"),
+            _stream_ptr(stream, N.device))
+    _check(st, "dt8_selfcheck_reciprocal")
     return out
 
 

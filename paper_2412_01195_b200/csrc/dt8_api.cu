@@ -61,6 +61,15 @@ divide_kernel(const float* __restrict__ s, const float* __restrict__ N, float* _
   }
 }
 
+// Diagnostic: the reciprocal the normalising division starts from.
+__global__ void __launch_bounds__(256)
+reciprocal_kernel(const float* __restrict__ N, float* __restrict__ out, int64_t n) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const Normaliser nz(N[i]);
+    out[i] = nz.fast ? nz.rN : 0.0f;
+  }
+}
 
 constexpr int kMaxDevices = 64;
 
@@ -370,6 +379,21 @@ int dt8_selfcheck_divide(const float* s, const float* N, int64_t n, float* out, 
   const int64_t ctas = (n + 255) / 256;
   const int grid = static_cast<int>(ctas < 8 * ctx.sm_count ? ctas : 8 * ctx.sm_count);
   divide_kernel<<<grid, 256, 0, ctx.stream>>>(s, N, out, n);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
+int dt8_selfcheck_reciprocal(const float* N, int64_t n, float* out, void* stream) {
+  if (n < 0) return DT8_ERR_INVALID_ARG;
+  if (n == 0) return DT8_OK;
+  if (!N || !out) return DT8_ERR_INVALID_ARG;
+  if (!aligned(N, 4) || !aligned(out, 4)) return DT8_ERR_ALIGNMENT;
+  LaunchCtx ctx;
+  int rc = ensure_device(&ctx, stream);
+  if (rc != DT8_OK) return rc;
+  const int64_t ctas = (n + 255) / 256;
+  const int grid = static_cast<int>(ctas < 8 * ctx.sm_count ? ctas : 8 * ctx.sm_count);
+  reciprocal_kernel<<<grid, 256, 0, ctx.stream>>>(N, out, n);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }

@@ -97,6 +97,28 @@ def test_quantize_follows_true_division(signed):
     quant_roundtrip_check(torch.from_numpy(x.ravel()), B, signed)
 
 
+def test_block_reciprocal_is_correctly_rounded_for_every_mantissa():
+    """The residual correction of Eq. quant1's division is exact only from the correctly rounded
+    reciprocal of the block maximum.  Inside 2^-76 .. 2^100 nothing in its computation overflows
+    or underflows, so the mantissa decides: all 2^23 of them, at the two ends and in the middle
+    of the range, against 1/N formed in binary64 and rounded once.  Outside the range, and for
+    N = 0, the routine reports that it takes the IEEE division (0)."""
+    man = np.arange(1 << 23, dtype=np.uint32)
+    for e in (-76, -75, -1, 0, 1, 64, 99):
+        N = (man | np.uint32((127 + e) << 23)).view(F)
+        got = dt8.dt8_selfcheck_reciprocal(torch.from_numpy(N).to(DEV)).cpu().numpy()
+        ref = (1.0 / N.astype(np.float64)).astype(F)
+        bad = np.nonzero(got != ref)[0]
+        assert bad.size == 0, (e, [float(x).hex() for x in N[bad[:4]]], got[bad[:4]], ref[bad[:4]])
+    edge = np.array([2.0 ** 100, 2.0 ** -76], F)
+    got = dt8.dt8_selfcheck_reciprocal(torch.from_numpy(edge).to(DEV)).cpu().numpy()
+    assert np.array_equal(got, np.array([2.0 ** -100, 2.0 ** 76], F))
+    outside = np.array([0.0, np.nextafter(F(2.0 ** 100), F(np.inf)), np.nextafter(F(2.0 ** -76), F(0)), 1e-40,
+                        np.inf, np.nan, 3e38], F)
+    got = dt8.dt8_selfcheck_reciprocal(torch.from_numpy(outside).to(DEV)).cpu().numpy()
+    assert np.array_equal(got, np.zeros(outside.size, F))
+
+
 def test_normalising_division_is_correctly_rounded():
     """Eq. quant1 divides: the kernels' reciprocal-and-correct routine must give the correctly
     rounded quotient for every |s| <= N.  The true quotient is formed in binary64 and rounded once
