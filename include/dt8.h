@@ -130,6 +130,17 @@ int dt8_selfcheck_divide(const float *s, const float *N, int64_t n, float *out, 
 int dt8_selfcheck_reciprocal(const float *N, int64_t n, float *out, void *stream);
 
 /*
+ * Diagnostic, device: out_i = the square root of x_i as the IEEE form of the Adam parameter
+ * update (Eq. adam, the root of the bias-corrected second moment) computes it when its operands
+ * are in range: a reciprocal-root approximation and one fused correction, which must be the
+ * correctly rounded root.  It depends on the mantissa and the parity of the exponent alone, so a
+ * test checks all 2^24 cases.  out_i = 0 for x_i outside 2^-80 .. 2^80, where the step uses the
+ * IEEE root instead.  No step, quantize or dequantize call uses it.
+ *   x  device, const float[n];   out  device, float[n]
+ */
+int dt8_selfcheck_root(const float *x, int64_t n, float *out, void *stream);
+
+/*
  * Diagnostic, device: out_i = s_i / d computed by the routine the IEEE form of the Adam parameter
  * update uses for Eq. adam's bias corrections m'/(1 - beta1^step), r'/(1 - beta2^step), whose
  * divisor is one number per launch: the host supplies the correctly rounded reciprocal of d and

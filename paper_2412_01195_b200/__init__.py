@@ -16,7 +16,7 @@ import torch
 
 __all__ = [
     "DT8Error", "lib_path", "load_library", "num_blocks",
-    "dt8_codebook", "dt8_state_bytes", "optimizer_state_bytes", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_selfcheck_reciprocal", "dt8_init",
+    "dt8_codebook", "dt8_state_bytes", "optimizer_state_bytes", "dt8_selfcheck_encode_host", "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_selfcheck_reciprocal", "dt8_selfcheck_root", "dt8_init",
     "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step", "dt8_adam_step", "dt8_sgd_step_multi",
     "dt8_adam_step_multi", "new_state", "shard_blocks", "PreparedTensorList",
@@ -37,7 +37,7 @@ _lib = None
 EXPORTS = (
     "dt8_status_string", "dt8_last_cuda_error", "dt8_codebook", "dt8_state_bytes",
     "dt8_selfcheck_encode_host",
-    "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_selfcheck_reciprocal", "dt8_init",
+    "dt8_selfcheck_divide", "dt8_selfcheck_divide_const", "dt8_selfcheck_reciprocal", "dt8_selfcheck_root", "dt8_init",
     "dt8_quantize_blockwise",
     "dt8_dequantize_blockwise", "dt8_sgd_step",
     "dt8_adam_step", "dt8_sgd_step_multi", "dt8_adam_step_multi",
@@ -81,6 +81,7 @@ def load_library() -> ctypes.CDLL:
     lib.dt8_selfcheck_divide.argtypes = [vp, vp, i64, vp, vp]
     lib.dt8_selfcheck_divide_const.argtypes = [vp, f32, i64, vp, vp]
     lib.dt8_selfcheck_reciprocal.argtypes = [vp, i64, vp, vp]
+    lib.dt8_selfcheck_root.argtypes = [vp, i64, vp, vp]
     lib.dt8_selfcheck_table_extents.argtypes = [vp, vp, vp, vp]
     lib.dt8_selfcheck_layout_fits.argtypes = [u32, i32, u32, i32]
     lib.dt8_init.argtypes = []
@@ -238,6 +239,18 @@ def dt8_selfcheck_reciprocal(N: torch.Tensor, out: Optional[torch.Tensor] = None
             _dev_tensor(N, torch.float32, "N"), N.numel(), _dev_tensor(out, torch.float32, "out"),
             _stream_ptr(stream, N.device))
     _check(st, "dt8_selfcheck_reciprocal")
+    return out
+
+
+def dt8_selfcheck_root(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Diagnostic: the square root of the fast IEEE Adam parameter update (0 outside its range)."""
+    if out is None:
+        out = torch.empty_like(x)
+    with _on_device(x.device):
+        st = load_library().dt8_selfcheck_root(
+            _dev_tensor(x, torch.float32, "x"), x.numel(), _dev_tensor(out, torch.float32, "out"),
+            _stream_ptr(stream, x.device))
+    _check(st, "dt8_selfcheck_root")
     return out
 
 

@@ -61,6 +61,16 @@ divide_kernel(const float* __restrict__ s, const float* __restrict__ N, float* _
   }
 }
 
+// Diagnostic: the square root of the fast IEEE parameter update.
+__global__ void __launch_bounds__(256)
+root_kernel(const float* __restrict__ x, float* __restrict__ out, int64_t n) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const float v = x[i];
+    out[i] = (v >= kFastRootMin && v <= kFastRootMax) ? sqrt_rn_inrange(v) : 0.0f;
+  }
+}
+
 // Diagnostic: the reciprocal the normalising division starts from.
 __global__ void __launch_bounds__(256)
 reciprocal_kernel(const float* __restrict__ N, float* __restrict__ out, int64_t n) {
@@ -238,7 +248,7 @@ AdamHyper make_adam_hyper(float lr, float beta1, float beta2, float eps, float w
   const ConstDivisor d1 = make_const_divisor(h.bc1), d2 = make_const_divisor(h.bc2);
   h.rbc1 = d1.rd;
   h.rbc2 = d2.rd;
-  h.const_div = (d1.usable && d2.usable) ? 1 : 0;
+  h.const_div = (d1.usable && d2.usable && eps <= kFastUpdateMaxEps) ? 1 : 0;
   h.neg_zero = -0.0f;
   return h;
 }
@@ -394,6 +404,21 @@ int dt8_selfcheck_reciprocal(const float* N, int64_t n, float* out, void* stream
   const int64_t ctas = (n + 255) / 256;
   const int grid = static_cast<int>(ctas < 8 * ctx.sm_count ? ctas : 8 * ctx.sm_count);
   reciprocal_kernel<<<grid, 256, 0, ctx.stream>>>(N, out, n);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? DT8_OK : cuda_fail(e);
+}
+
+int dt8_selfcheck_root(const float* x, int64_t n, float* out, void* stream) {
+  if (n < 0) return DT8_ERR_INVALID_ARG;
+  if (n == 0) return DT8_OK;
+  if (!x || !out) return DT8_ERR_INVALID_ARG;
+  if (!aligned(x, 4) || !aligned(out, 4)) return DT8_ERR_ALIGNMENT;
+  LaunchCtx ctx;
+  int rc = ensure_device(&ctx, stream);
+  if (rc != DT8_OK) return rc;
+  const int64_t ctas = (n + 255) / 256;
+  const int grid = static_cast<int>(ctas < 8 * ctx.sm_count ? ctas : 8 * ctx.sm_count);
+  root_kernel<<<grid, 256, 0, ctx.stream>>>(x, out, n);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? DT8_OK : cuda_fail(e);
 }

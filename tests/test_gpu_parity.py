@@ -119,6 +119,45 @@ def test_block_reciprocal_is_correctly_rounded_for_every_mantissa():
     assert np.array_equal(got, np.zeros(outside.size, F))
 
 
+def test_fast_root_is_correctly_rounded_for_every_mantissa_and_parity():
+    """The IEEE form of Eq. adam's parameter update takes sqrt(r'/bc2); inside 2^-80 .. 2^80 the
+    kernel forms it from a reciprocal-root approximation and one correction.  The outcome depends
+    on the mantissa and on the parity of the exponent only: all 2^24 cases at the ends and in the
+    middle of the range, against the root formed in binary64 and rounded once (a binary64 root of
+    a binary32 number is never close enough to a binary32 rounding boundary for the second rounding
+    to matter).  Outside the range the routine reports 0 (the step then uses the IEEE root)."""
+    man = np.arange(1 << 23, dtype=np.uint32)
+    for e in (-80, -79, -1, 0, 1, 2, 79):
+        x = (man | np.uint32((127 + e) << 23)).view(F)
+        got = dt8.dt8_selfcheck_root(torch.from_numpy(x).to(DEV)).cpu().numpy()
+        ref = np.sqrt(x.astype(np.float64)).astype(F)
+        bad = np.nonzero(got != ref)[0]
+        assert bad.size == 0, (e, [float(v).hex() for v in x[bad[:4]]], got[bad[:4]], ref[bad[:4]])
+    edge = np.array([2.0 ** 80, 2.0 ** -80], F)
+    assert np.array_equal(dt8.dt8_selfcheck_root(torch.from_numpy(edge).to(DEV)).cpu().numpy(),
+                          np.array([2.0 ** 40, 2.0 ** -40], F))
+    outside = np.array([0.0, -1.0, np.nextafter(F(2.0 ** 80), F(np.inf)), np.nextafter(F(2.0 ** -80), F(0)),
+                        np.inf, np.nan], F)
+    assert np.array_equal(dt8.dt8_selfcheck_root(torch.from_numpy(outside).to(DEV)).cpu().numpy(),
+                          np.zeros(outside.size, F))
+
+
+def test_reciprocal_and_correct_division_for_quotients_of_any_size():
+    """The same reciprocal-and-correct division serves Eq. adam's m-hat / (sqrt(r-hat) + eps) in
+    the IEEE parameter update, where the dividend may exceed the divisor: dividends 2^-80 .. 2^80
+    over divisors 2^-40 .. 2^46 (the ranges the step guarantees), against the quotient formed in
+    binary64 and rounded once."""
+    rng = np.random.default_rng(11)
+    M = 1 << 23
+    d = (rng.uniform(1, 2, M) * 2.0 ** rng.integers(-40, 46, M)).astype(F)
+    a = (rng.uniform(1, 2, M) * 2.0 ** rng.integers(-80, 80, M) * rng.choice([-1.0, 1.0], M)).astype(F)
+    # special mantissas of the divisor
+    d[:1 << 20] = ((rng.integers(0, 1 << 23, 1 << 20).astype(np.uint32) | np.uint32(0x7FFF00)) & np.uint32(0x7FFFFF) | np.uint32(0x3F800000)).view(F)
+    got = dt8.dt8_selfcheck_divide(torch.from_numpy(a).to(DEV), torch.from_numpy(d).to(DEV)).cpu().numpy()
+    ref = (a.astype(np.float64) / d.astype(np.float64)).astype(F)
+    assert np.array_equal(got, ref)
+
+
 def test_normalising_division_is_correctly_rounded():
     """Eq. quant1 divides: the kernels' reciprocal-and-correct routine must give the correctly
     rounded quotient for every |s| <= N.  The true quotient is formed in binary64 and rounded once
