@@ -88,8 +88,8 @@ DT8_HD uint32_t byte_perm(uint32_t x, uint32_t y, uint32_t sel) {
 // (sub.cc / subc): two instructions, no predicate and no select.
 DT8_HD uint32_t below_by_borrow(uint32_t entry, uint32_t x) {
 #if defined(__CUDA_ARCH__)
-  uint32_t diff, r;
-  asm("{\n\tsub.cc.u32 %0, %3, %2;\n\tsubc.u32 %1, %2, 0;\n\t}" : "=r"(diff), "=r"(r) : "r"(entry), "r"(x));
+  uint32_t r;
+  asm("{\n\t.reg .b32 diff;\n\tsub.cc.u32 diff, %2, %1;\n\tsubc.u32 %0, %1, 0;\n\t}" : "=r"(r) : "r"(entry), "r"(x));
   return r;
 #else
   return entry - (x < entry ? 1u : 0u);
