@@ -49,6 +49,56 @@ def test_ieee_parameter_paths(case, gdtype, B):
     st.check(exact_params=True)
 
 
+@pytest.mark.parametrize("eps", [0.0, 1e-8, 3.0e13, 4.0e13, 1e30])
+def test_ieee_update_across_the_edges_of_its_fast_range(eps):
+    """The IEEE parameter update replaces the library root and divisions by corrected
+    approximations only while every moment of a thread lies in 2^-60 .. 2^60 and eps is at most
+    2^45 (3.5e13); blocks of gradients from 1e-30 to 1e15 put moments below, inside, on both sides
+    of the edges of, and above that range, and the eps values sit on both sides of its limit.  The
+    parameters must equal the checker's bit for bit wherever the update ran."""
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=eps, weight_decay=1e-3)
+    B = 2048
+    scales = [1e-30, 1e-15, 1e-12, 1e-9, 3e-9, 1e-7, 1e-3, 1.0, 1e3, 1e8, 1e10, 3e10, 1e11, 1e15]
+    if eps == 0.0:
+        scales[0] = scales[1] = 1e-12     # a squared gradient that underflows to 0 would divide by zero
+    n = len(scales) * B + 77
+    w0 = synth.normal(n, 1.0, 1250)
+    scale = torch.ones(n)
+    for k, s in enumerate(scales):
+        scale[k * B:(k + 1) * B] = s
+    # one block mixes magnitudes inside a thread's sixteen values
+    scale[7 * B:8 * B:5] = 1e-12
+    st = AdamState(w0 * scale, B)
+    for t in range(1, 5):
+        st.step(synth.fresh_grad(n, 125, t) * scale, t, hp, BC)
+    st.check(exact_params=True)
+
+
+@pytest.mark.parametrize("B", [256, 2048])
+def test_states_of_very_small_and_very_large_gradients(B):
+    """Blocks whose maxima leave the range of the reciprocal-and-correct normalisation (below
+    2^-76, above 2^100) take the IEEE division, a block of zeros stays zeros, and both can meet in
+    one block: a gradient of 1e-30 gives a first moment of 1e-31 and a second moment that
+    underflows to exactly 0.  Codes and maxima must equal the checker's; SGD likewise."""
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    scales = [1e-30, 1e-25, 1e-20, 1e-12, 1.0, 1e12, 1e16, 1e18]
+    n = len(scales) * B + 5
+    scale = torch.ones(n)
+    for k, s in enumerate(scales):
+        scale[k * B:(k + 1) * B] = s
+    st = AdamState(synth.normal(n, 0.02, 1260), B)
+    sg = SgdState(synth.normal(n, 0.02, 1261), B)
+    sg_small = SgdState(synth.normal(n, 0.02, 1262), B)
+    for t in range(1, 5):
+        g = synth.fresh_grad(n, 126, t) * scale
+        st.step(g, t, hp)
+        sg.step(g * 1e14, t, dict(lr=1e-3, momentum=0.9, weight_decay=0.0))
+        sg_small.step(g, t, dict(lr=1e-3, momentum=0.9, weight_decay=0.0))
+    st.check()
+    sg.check()
+    sg_small.check()
+
+
 def test_coupled_decay_from_the_zero_state_with_zero_gradients():
     """All-zero groups (dividend 0) take the IEEE division inside the IEEE path."""
     hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
