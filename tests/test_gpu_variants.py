@@ -81,7 +81,7 @@ def test_states_of_very_small_and_very_large_gradients(B):
     one block: a gradient of 1e-30 gives a first moment of 1e-31 and a second moment that
     underflows to exactly 0.  Codes and maxima must equal the checker's; SGD likewise."""
     hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
-    scales = [1e-30, 1e-25, 1e-20, 1e-12, 1.0, 1e12, 1e16, 1e18]
+    scales = [1e-41, 1e-38, 1e-36, 1e-30, 1e-25, 1e-20, 1e-12, 1.0, 1e12, 1e16, 1e18]
     n = len(scales) * B + 5
     scale = torch.ones(n)
     for k, s in enumerate(scales):
