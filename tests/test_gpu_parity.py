@@ -50,6 +50,25 @@ def test_quantize_dequantize_sizes_and_tails(B, signed):
 
 
 @pytest.mark.parametrize("signed", [True, False])
+@pytest.mark.parametrize("B", [256, 2048])
+def test_quantize_blocks_of_every_magnitude(B, signed):
+    """Block maxima from subnormal to close to the largest binary32 number, with the edges of the
+    range of the reciprocal-and-correct division (2^-76 = 1.3e-23, 2^100 = 1.3e30) on both sides,
+    a block of zeros, and blocks that mix a large maximum with values far below the smallest code."""
+    scales = [1e-44, 1e-41, 1e-39, 1e-37, 1e-30, 1.2e-23, 1.4e-23, 1e-10, 1.0, 1e10, 1.2e30, 1.4e30,
+              1e34, 3e37, 0.0]
+    n = len(scales) * B
+    x = synth.laplace_outliers(n, seed=350).clamp(-8, 8)
+    for k, s in enumerate(scales):
+        x[k * B:(k + 1) * B] *= s
+    x[4 * B + 5] = 1e-5        # values 25 decades below the block maximum
+    x[9 * B:10 * B:3] *= 1e-30
+    if not signed:
+        x = x.abs()
+    quant_roundtrip_check(x, B, signed)
+
+
+@pytest.mark.parametrize("signed", [True, False])
 def test_quantize_sweep_configuration(signed):
     """Configuration 4 at its smaller sizes: Laplace(0,1) with 1e-3 outliers x100 (the 128M size is
     covered by sampled blocks in the full-size test)."""
