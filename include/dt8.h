@@ -215,7 +215,9 @@ int dt8_sgd_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *
  * and square root (relative error ~2e-7 of the update term; when eps*sqrt(bc2) < 1e-12 the forms
  * of these instructions that keep subnormal numbers are used, so that a tiny second moment is not
  * flushed to zero).  With coupled decay, where p feeds the states, and for a learning rate outside
- * 1e-20 .. 1e20, it is evaluated with IEEE operations and is bit-reproducible against a plain
+ * 1e-20 .. 1e20, every written operation is one correctly rounded binary32 operation (the
+ * divisions and the root by the IEEE instructions, or inside their tested ranges by corrected
+ * approximations with the same results), so that the update is bit-reproducible against a plain
  * binary32 evaluation.
  */
 int dt8_adam_step(float *p, const void *g, int g_dtype, uint8_t *m_codes, float *m_absmax,
