@@ -105,3 +105,76 @@ def test_random_quantize_configurations(chunk):
         assert np.array_equal(to_np(absmax), ra), seed
         assert np.array_equal(to_np(codes), rc), seed
         assert np.array_equal(to_np(out).view(np.uint32), oracle.dequantize_blockwise(rc, ra, B, signed).view(np.uint32)), seed
+
+
+@pytest.mark.parametrize("chunk", range(3))
+def test_random_pointer_lists(chunk):
+    """Lists of 1 to 300 tensors of random sizes (empty and tiny ones, whole blocks, ragged tails),
+    Adam or SGD, either gradient type: the pointer-list launch equals the checker tensor by tensor."""
+    for seed in range(9900 + 8 * chunk, 9900 + 8 * (chunk + 1)):
+        rng = np.random.default_rng(seed)
+        B = int(rng.choice(dt8.BLOCK_SIZES))
+        count = int(rng.choice([1, 2, 17, 120, 257, 300]))
+        kinds = rng.integers(0, 4, count)
+        sizes = [0 if k == 0 and rng.random() < 0.2 else
+                 int(rng.integers(1, 65)) if k <= 1 else
+                 int(rng.integers(1, 4)) * B if k == 2 else
+                 int(rng.integers(1, 3 * B)) for k in kinds]
+        gdt = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+        adam = bool(rng.random() < 0.6)
+        steps = int(rng.integers(1, 4))
+        ws = [torch.from_numpy((rng.standard_normal(n) * 0.05).astype(F)) for n in sizes]
+        if adam:
+            hp = (float(10 ** rng.uniform(-4, -2)), 0.9, 0.999, 1e-8, float(rng.choice([0.0, 0.01])))
+            flags = int(rng.choice([1, 3, 3]))
+            sts = [AdamState(w, B) for w in ws]
+        else:
+            hp = (float(10 ** rng.uniform(-3, -1)), 0.9, float(rng.choice([0.0, 1e-4])))
+            sts = [SgdState(w, B) for w in ws]
+        for t in range(1, steps + 1):
+            gs = [torch.from_numpy((rng.standard_normal(n) * 0.01).astype(F)).to(gdt) for n in sizes]
+            gg = [g.cuda() for g in gs]
+            if adam:
+                dt8.dt8_adam_step_multi([s.w_gpu for s in sts], gg, [s.mc_gpu for s in sts], [s.ma_gpu for s in sts],
+                                        [s.rc_gpu for s in sts], [s.ra_gpu for s in sts], *hp, t, B, flags)
+                for s, g in zip(sts, gs):
+                    oracle.adam_step(s.w, to_np(g), s.mc, s.ma, s.rc, s.ra, *hp, t, B, flags)
+            else:
+                dt8.dt8_sgd_step_multi([s.w_gpu for s in sts], gg, [s.mc_gpu for s in sts], [s.ma_gpu for s in sts],
+                                       *hp, t, B)
+                for s, g in zip(sts, gs):
+                    oracle.sgd_step(s.w, to_np(g), s.mc, s.ma, *hp, t, B)
+        for s in sts:
+            if adam:
+                s.check(rel=1e-5, exact_params=not (flags & dt8.DT8_ADAM_DECOUPLED_WD) and hp[4] != 0.0)
+            else:
+                s.check()
+
+
+def test_random_reversible_kernel_shapes():
+    """Coupling halves and the invertible down-sampling on random N x C x F x T shapes (rows of any
+    even length, so that every vector width and the small-plane path are met) against the checker,
+    bit for bit, and each followed by its inverse."""
+    from oracle import rev as orev
+    from paper_2412_01195_b200 import rev
+    for seed in range(9950, 9990):
+        rng = np.random.default_rng(seed)
+        N, C = int(rng.integers(1, 5)), 2 * int(rng.integers(1, 7))
+        Fd, T = 2 * int(rng.integers(1, 13)), 2 * int(rng.integers(1, 60))
+        x = rng.standard_normal((N, C, Fd, T)).astype(F)
+        t = rng.standard_normal((N, C // 2, Fd, T)).astype(F)
+        which = int(rng.integers(0, 2))
+        xg, tg = torch.from_numpy(x).cuda(), torch.from_numpy(t).cuda()
+        yg = xg.clone()
+        rev.dt8_rev_coupling_forward(xg, tg, yg, which)
+        y = x.copy()
+        orev.couple_half(x, t, y, which, +1)
+        assert np.array_equal(to_np(yg), y), seed
+        back = yg.clone()
+        rev.dt8_rev_coupling_inverse(yg, tg, back, which)
+        ref_back = y.copy()
+        orev.couple_half(y, t, ref_back, which, -1)
+        assert np.array_equal(to_np(back), ref_back), seed
+        deep = rev.dt8_rev_space_to_depth(xg)
+        assert np.array_equal(to_np(deep), orev.space_to_depth(x)), seed
+        assert torch.equal(rev.dt8_rev_depth_to_space(deep), xg), seed
